@@ -1,0 +1,184 @@
+/*
+ * libfcp — the single-GPU hot path of Flexible Context Parallelism (FCP) for B200 (sm_100a).
+ *
+ * Varlen causal attention, forward and backward, over a packed batch of sequences of very
+ * different lengths.  Every sequence carries its own context-parallel (CP) degree d (any positive
+ * integer, Sec. 4.2 "any positive integer parallelism degree"); it is cut evenly along the sequence
+ * dimension (Sec. 4.3) into 2d load-balanced chunks, and every (Q chunk, KV chunk) block pair that
+ * a virtual rank of a ring-style CP group (Sec. 3.2) would compute is executed on one GPU, giving
+ * partial outputs and log-sum-exps that a merge kernel combines exactly.  The per-batch strategy
+ * search of Sec. 4.4 (best-fit-decreasing grouping + 2-D dynamic programme, Eq. 7, Algorithm 1)
+ * runs on the host and emits the per-sequence degrees.
+ *
+ * Conventions
+ *   - Plain C ABI.  Every function returns an int status (FCP_OK == 0, negative = error) and never
+ *     throws or aborts.  fcp_status_string() names a status.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global memory of the
+ *     current device.  The caller owns every buffer it passes; the library owns only fcp_plan
+ *     objects (host tables plus, after fcp_plan_upload, a device copy of them).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Compute calls only
+ *     enqueue work on it; they do not synchronise and do not allocate device memory.
+ *   - Tensors are packed token-major ("THD"), row-major, bf16:
+ *         q, o, d_o, dq : [T][hq][D]        k, v, dk, dv : [T][hkv][D]
+ *     T = total tokens of the batch, D = head_dim in {64, 128}, hq % hkv == 0; query head h reads
+ *     KV head h / (hq/hkv).  lse is fp32 [T][hq], natural log of the sum of exp(scaled scores).
+ *   - Limits: T and the number of partial rows R are < 2^31; device byte offsets are 64-bit.
+ */
+#ifndef FCP_H_
+#define FCP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FCP_OK                 0
+#define FCP_ERR_INVALID_ARG   (-1)   /* NULL pointer, non-positive size, bad enum                    */
+#define FCP_ERR_INFEASIBLE    (-2)   /* planner: the minimum degrees need more than N ranks          */
+#define FCP_ERR_UNSUPPORTED   (-3)   /* head_dim not 64/128, hq % hkv != 0, degree > FCP_MAX_DEGREE   */
+#define FCP_ERR_WORKSPACE     (-4)   /* a caller-provided workspace is too small                      */
+#define FCP_ERR_CUDA          (-5)   /* a CUDA runtime/driver call failed, or no usable device        */
+#define FCP_ERR_TIMEOUT       (-6)   /* a bounded device-side wait expired (reported by fcp_last_device_status) */
+#define FCP_ERR_NOT_UPLOADED  (-7)   /* compute call on a plan without a device copy                  */
+
+#define FCP_MAX_DEGREE 64            /* largest CP degree of one sequence                             */
+
+typedef struct fcp_plan fcp_plan;
+
+/* Shape of the attention problem.  scale <= 0 selects 1/sqrt(head_dim) (Sec. 3.1, Eq. 1). */
+typedef struct fcp_params {
+  int32_t hq;        /* query heads                                  */
+  int32_t hkv;       /* key/value heads (hq % hkv == 0)               */
+  int32_t head_dim;  /* 64 or 128                                     */
+  float   scale;     /* softmax scale; <= 0 means 1/sqrt(head_dim)    */
+} fcp_params;
+
+/* Profiled coefficients of the cost model, Eqs. 4-6 (Sec. 4.3).  eta is the per-sequence mask
+ * efficiency factor (host array of B doubles) or NULL for all-causal (eta = 0). */
+typedef struct fcp_cost_coeffs {
+  double alpha1, alpha2, alpha3, beta1, beta2, v;
+  const double* eta;
+} fcp_cost_coeffs;
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_plan_strategy — host only.  Sec. 4.4: stage 1 groups the B sequences into K' atomic groups
+ * by best-fit-decreasing under the per-rank activation budget E - M_ms (Eq. 3; a sequence that
+ * opens a group fixes d_min = ceil(len*M_token / (E - M_ms))); stage 2 is the 2-D dynamic programme
+ * DP[i][j] = min_d max(DP[i-1][j-d], T(G_i, d)) of Eq. 7 / Algorithm 1 with strict-less updates,
+ * backtracked from DP[K'][N], so the degrees add up to exactly N.  T(G, d) is Eq. 6 with the
+ * per-rank reading of Eqs. 4-5: compute terms divided by d, ring communication only when d > 1.
+ *   in : seqlens[B] (host), N ranks, E, M_token, M_ms, coefficients
+ *   out: group_of[B] (group index of each sequence, groups in creation order), cp_degree[B]
+ *        (degree of the sequence's group), *n_groups, *makespan = DP[K'][N]; any may be NULL.
+ * Errors: FCP_ERR_INVALID_ARG (NULL inputs, B <= 0, N <= 0, E <= M_ms, non-positive length or
+ * M_token), FCP_ERR_INFEASIBLE (sum of d_min > N), FCP_ERR_UNSUPPORTED (N > FCP_MAX_DEGREE).
+ */
+int fcp_plan_strategy(const int32_t* seqlens, int32_t B, int32_t N, double E, double M_token,
+                      double M_ms, const fcp_cost_coeffs* coeffs, int32_t* group_of,
+                      int32_t* cp_degree, int32_t* n_groups, double* makespan);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_plan_blocks — host only.  Builds the block plan of a packed batch: for each sequence of
+ * length L and degree d the 2d+1 chunk bounds floor(c*L/(2d)) ("evenly into chunks", Sec. 4.3),
+ * and for each virtual rank r (owning chunks r and 2d-1-r) and ring step s (holding the KV of
+ * rank (r-s) mod d) the causally needed block pairs; pairs with an empty chunk are dropped.  One
+ * partial-output slot per (Q chunk, rank, step).  Also derives the kernels' work lists.
+ *   in : seqlens[B], cp_degrees[B] (host), params
+ *   out: *plan (release with fcp_plan_destroy)
+ * Errors: INVALID_ARG (NULL, B <= 0, length <= 0, degree <= 0, T or R >= 2^31),
+ * UNSUPPORTED (head_dim, head ratio, degree > FCP_MAX_DEGREE).
+ */
+int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
+                    const fcp_params* params, fcp_plan** plan);
+
+/* Tables readable through fcp_plan_get.  All are int32, row-major, host memory owned by the plan.
+ * Rows are in the canonical order (sequence, rank, step, q_chunk, kv_chunk).                     */
+#define FCP_TABLE_CU_SEQLENS    0  /* [B+1]                     packed-token offsets of the sequences */
+#define FCP_TABLE_CHUNK_OFFSET  1  /* [B+1]                     offsets into CHUNK_BOUNDS             */
+#define FCP_TABLE_CHUNK_BOUNDS  2  /* [sum(2d+1)]               packed-token chunk bounds             */
+#define FCP_TABLE_PAIRS         3  /* [n_pairs][6]  seq, rank, step, q_chunk, kv_chunk, kind (0 FULL, 1 DIAG) */
+#define FCP_TABLE_ITEMS         4  /* [n_items][8]  seq, rank, step, q_chunk, slot, part_row0, n_pairs, first_pair */
+#define FCP_TABLE_SLOT_OFFSET   5  /* [n_chunks+1]              offsets into SLOT_ROWS, chunks in (seq, chunk) order */
+#define FCP_TABLE_SLOT_ROWS     6  /* [sum n_slots]             part_row0 of each slot of each chunk  */
+#define FCP_TABLE_FWD_UNITS     7  /* [n_fwd_units][16]         derived; execution order, not canonical */
+#define FCP_TABLE_BWD_UNITS     8  /* [n_bwd_units][8]          derived                               */
+#define FCP_TABLE_BWD_QRANGES   9  /* [n_bwd_qranges][4]        derived                               */
+#define FCP_TABLE_MERGE_UNITS  10  /* [n_merge_units][4]        derived                               */
+
+/* fcp_plan_get: *host_ptr = first element of the table, *count = number of int32 elements. */
+int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count);
+
+/* Scalar facts about a plan: which in {0: T, 1: R (partial rows), 2: n_pairs, 3: n_items,
+ * 4: n_fwd_units, 5: n_bwd_units, 6: n_merge_units, 7: B}.                                       */
+int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value);
+
+/* Bytes the caller must provide: o_partial = R*heads_per_pass*D*4, lse_partial = R*heads_per_pass*4,
+ * bwd_scratch (all hq heads at once) for fcp_attn_bwd.  Any output pointer may be NULL.          */
+int fcp_plan_workspace_bytes(const fcp_plan* plan, int32_t heads_per_pass, int64_t* o_partial_bytes,
+                             int64_t* lse_partial_bytes, int64_t* bwd_scratch_bytes);
+
+/* Copies the plan's work tables to the current device (the only device allocation the library
+ * makes; freed by fcp_plan_destroy).  Must precede the compute calls.  Synchronous.              */
+int fcp_plan_upload(fcp_plan* plan, void* stream);
+int fcp_plan_destroy(fcp_plan* plan);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_attn_fwd — device.  For every item of the plan and every query head h in
+ * [head_begin, head_begin+head_count): softmax(q k^T * scale) v (Eq. 1) restricted to the item's
+ * KV ranges with the causal mask k_pos <= q_pos, as a NORMALISED partial output and its
+ * log-sum-exp:
+ *     o_partial  [R][head_count][D] fp32,   lse_partial [R][head_count] fp32
+ * Row r of an item = part_row0 + (token - first token of its Q chunk).
+ * q, k, v: device bf16.  Asynchronous on `stream`.
+ */
+int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v,
+                 int32_t head_begin, int32_t head_count, float* o_partial, float* lse_partial,
+                 void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_lse_merge — device.  Exact combination of the slots of every (token, head):
+ *     LSE = m + log sum_s exp(lse_s - m),  o = sum_s exp(lse_s - LSE) * o_s     (m = max_s lse_s)
+ * (the re-association of the softmax sum implied by ring-style CP, Sec. 3.2).
+ * Writes o[T][hq][D] bf16 and lse[T][hq] fp32 for heads [head_begin, head_begin+head_count); the
+ * partial buffers have head_count heads (the layout fcp_attn_fwd wrote).
+ */
+int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
+                  int32_t head_begin, int32_t head_count, void* o, float* lse, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_attn_bwd — device.  Gradients of Eq. 1 with the causal mask, evaluated over the plan's
+ * block pairs grouped by KV chunk: with P = exp(S*scale - LSE), delta_i = dO_i . O_i,
+ *     dV = P^T dO,  dP = dO V^T,  dS = P o (dP - delta),  dQ = scale dS K,  dK = scale dS^T Q,
+ * dK/dV summed over the hq/hkv query heads of a KV head.  o, lse are the merged forward results.
+ * scratch: device buffer of at least bwd_scratch_bytes (fcp_plan_workspace_bytes); its contents
+ * need not be initialised.  dq/dk/dv: device bf16 outputs (every element is written).
+ */
+int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                 const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* scratch,
+                 int64_t scratch_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_attn_fwd_bwd_host — the whole path from HOST buffers: copies q, k, v, d_o to the device,
+ * runs fcp_attn_fwd (in head passes that fit the workspace), fcp_lse_merge and fcp_attn_bwd, and
+ * copies o, lse, dq, dk, dv back.  `workspace` is a caller-owned DEVICE buffer of
+ * `workspace_bytes` >= fcp_host_workspace_bytes(plan); host pointers should be pinned for the
+ * copies to be asynchronous.  Synchronises `stream` before returning.
+ */
+int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes);
+int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host,
+                          const void* v_host, const void* d_o_host, void* o_host, float* lse_host,
+                          void* dq_host, void* dk_host, void* dv_host, void* workspace,
+                          int64_t workspace_bytes, void* stream);
+
+/* Device-side status word of the last kernels run with this plan (0 = fine; FCP_ERR_TIMEOUT if a
+ * bounded wait inside a kernel expired).  Synchronises the device.                               */
+int fcp_last_device_status(const fcp_plan* plan, int32_t* status);
+
+const char* fcp_status_string(int status);
+const char* fcp_last_error_message(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FCP_H_ */

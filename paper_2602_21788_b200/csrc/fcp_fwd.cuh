@@ -1,0 +1,334 @@
+// Forward attention over the block plan (Eq. 1 of the paper restricted to an item's KV ranges,
+// causal mask k_pos <= q_pos), one persistent grid for all virtual ranks of all sequences.
+//
+// Work unit = (two adjacent 128-row Q tiles of one plan item, one query head).  Roles per CTA:
+//   warp 0        TMA producer: Q tiles and the K/V tile ring (128-byte swizzled boxes)
+//   warp 1        UMMA issuer:  S = Q K^T into TMEM, O += P V with P read from TMEM
+//   warps 2..5    softmax for Q tile 0 (one thread per query row), epilogue
+//   warps 6..9    softmax for Q tile 1
+// TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each (D = 128); bf16 P overwrites the
+// first 64 columns of its S.  While one tile's softmax runs on the CUDA cores the tensor core works
+// on the other tile, so the two Q tiles share every K/V tile that is staged.
+#pragma once
+#include "fcp_plan.hpp"
+#include "sm100_ptx.cuh"
+
+namespace fcp {
+
+constexpr int FWD_THREADS = 320;
+constexpr int FWD_KV_SLOTS = 4;
+
+template <int D>
+struct FwdSmem {
+  static constexpr int Q_TILE_BYTES = 128 * D * 2;
+  static constexpr int KV_TILE_BYTES = 128 * D * 2;
+  static constexpr int Q_OFF = 0;
+  static constexpr int KV_OFF = 2 * Q_TILE_BYTES;
+  static constexpr int BAR_OFF = KV_OFF + FWD_KV_SLOTS * KV_TILE_BYTES;
+  // barriers: q_full[2] q_empty[2] kv_full[S] kv_empty[S] s_full[2] p_full[2] o_final[2] o_empty[2]
+  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 8;
+  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;   // tmem base (4 B), abort flag (4 B)
+  static constexpr int TOTAL = MISC_OFF + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;          // slack to align the base to 1024 B
+};
+
+struct FwdArgs {
+  const int32_t* units;   // [n_units][16]
+  int32_t n_units;
+  int32_t head_begin, head_count, hq, hkv;
+  float scale_log2;       // softmax scale * log2(e)
+  float* o_partial;       // [R][head_count][D]
+  float* lse_partial;     // [R][head_count]
+  int32_t* status;        // [4]
+};
+
+template <int D>
+__global__ void __launch_bounds__(FWD_THREADS, 1)
+fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+               const __grid_constant__ CUtensorMap tm_v, const FwdArgs a) {
+  using SM = FwdSmem<D>;
+  constexpr int KBLK = D / 64;                 // 64-element (128-byte) column blocks per row
+  constexpr uint32_t BLK_BYTES = 128 * 128;    // one [128 rows][64] swizzled block
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t S_COL0 = 0, O_COL0 = 256; // S stage s at 128*s, O stage s at 256 + 128*s
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar0 = sbase + SM::BAR_OFF;
+  auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  const int B_QFULL = 0, B_QEMPTY = 2, B_KVFULL = 4, B_KVEMPTY = 4 + FWD_KV_SLOTS,
+            B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6;
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
+  volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
+  const WaitCtx wctx{abort_flag, a.status};
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    *abort_flag = 0;
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(BAR(B_QFULL + i), 1);
+      mbar_init(BAR(B_QEMPTY + i), 1);
+      mbar_init(BAR(B_SFULL + i), 1);
+      mbar_init(BAR(B_PFULL + i), 128);
+      mbar_init(BAR(B_OFINAL + i), 1);
+      mbar_init(BAR(B_OEMPTY + i), 128);
+    }
+    for (int i = 0; i < FWD_KV_SLOTS; ++i) {
+      mbar_init(BAR(B_KVFULL + i), 1);
+      mbar_init(BAR(B_KVEMPTY + i), 1);
+    }
+    fence_mbar_init();
+    prefetch_tmap(&tm_q);
+    prefetch_tmap(&tm_k);
+    prefetch_tmap(&tm_v);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32((const void*)tmem_slot), TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  const int64_t n_work = (int64_t)a.n_units * a.head_count;
+  const int g = a.hq / a.hkv;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kv_it = 0, qcnt[2] = {0, 0};
+      bool ok = true;
+      for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+        const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+        const int h = a.head_begin + (int)(w % a.head_count);
+        const int hk = h / g;
+        const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
+        const int q_row0 = __ldg(U + FU_Q_ROW0);
+        for (int s = 0; s < 2 && ok; ++s) {
+          if (nt[s] == 0) continue;
+          ok = mbar_wait(BAR(B_QEMPTY + s), (qcnt[s] & 1) ^ 1, wctx, 10 + s);
+          if (!ok) break;
+          mbar_expect_tx(BAR(B_QFULL + s), SM::Q_TILE_BYTES);
+          for (int kb = 0; kb < KBLK; ++kb)
+            tma_load_3d(sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES + kb * BLK_BYTES, &tm_q, BAR(B_QFULL + s), kb * 64, h,
+                        q_row0 + s * 128);
+          ++qcnt[s];
+        }
+        const int n_max = max(nt[0], nt[1]);
+        const int nr0 = __ldg(U + FU_NT_RANGE0);
+        const int kv0 = __ldg(U + FU_KV0_BEGIN), kv1 = __ldg(U + FU_KV1_BEGIN);
+        for (int j = 0; j < n_max && ok; ++j) {
+          const int row = j < nr0 ? kv0 + j * 128 : kv1 + (j - nr0) * 128;
+          for (int t = 0; t < 2; ++t) {   // t = 0: K tile, t = 1: V tile
+            const uint32_t slot = kv_it % FWD_KV_SLOTS;
+            ok = mbar_wait(BAR(B_KVEMPTY + slot), ((kv_it / FWD_KV_SLOTS) & 1) ^ 1, wctx, 12);
+            if (!ok) break;
+            mbar_expect_tx(BAR(B_KVFULL + slot), SM::KV_TILE_BYTES);
+            for (int kb = 0; kb < KBLK; ++kb)
+              tma_load_3d(sbase + SM::KV_OFF + slot * SM::KV_TILE_BYTES + kb * BLK_BYTES, t == 0 ? &tm_k : &tm_v,
+                          BAR(B_KVFULL + slot), kb * 64, hk, row);
+            ++kv_it;
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ UMMA issuer
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = make_idesc(128, 128, 0, 0);
+      constexpr uint32_t IDESC_PV = make_idesc(128, D, 0, 1);
+      uint32_t kv_it = 0, qcnt[2] = {0, 0}, pcnt[2] = {0, 0}, ocnt[2] = {0, 0};
+      bool ok = true;
+      for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+        const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+        const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
+        const int n_max = max(nt[0], nt[1]);
+        for (int s = 0; s < 2 && ok; ++s)
+          if (nt[s] > 0) {
+            ok = mbar_wait(BAR(B_QFULL + s), qcnt[s] & 1, wctx, 20 + s);
+            ++qcnt[s];
+          }
+        for (int j = 0; j <= n_max && ok; ++j) {
+          // ring positions: K_j at kv_it + 2j, V_{j-1} at kv_it + 2j - 1
+          const uint32_t itK = kv_it + 2 * j, itV = kv_it + 2 * j - 1;
+          const uint32_t slotK = itK % FWD_KV_SLOTS, slotV = itV % FWD_KV_SLOTS;
+          if (j >= 1) ok = mbar_wait(BAR(B_KVFULL + slotV), (itV / FWD_KV_SLOTS) & 1, wctx, 22);
+          if (ok && j < n_max) ok = mbar_wait(BAR(B_KVFULL + slotK), (itK / FWD_KV_SLOTS) & 1, wctx, 23);
+          if (!ok) break;
+          for (int s = 0; s < 2 && ok; ++s) {
+            if (j >= 1 && j - 1 < nt[s]) {
+              // O_s (+)= P_s(j-1) V_{j-1}
+              if (j == 1) {
+                ok = mbar_wait(BAR(B_OEMPTY + s), (ocnt[s] & 1) ^ 1, wctx, 24 + s);
+                ++ocnt[s];
+                if (!ok) break;
+              }
+              ok = mbar_wait(BAR(B_PFULL + s), pcnt[s] & 1, wctx, 26 + s);
+              ++pcnt[s];
+              if (!ok) break;
+              tc_fence_after();
+              const uint32_t vbase = sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES;
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {   // 128 keys = 8 steps of K = 16
+                const uint64_t bdesc = make_sdesc(vbase + k * 2048, BLK_BYTES, 1024);
+                umma_ts(tmem + O_COL0 + s * 128, tmem + S_COL0 + s * 128 + k * 8, bdesc, IDESC_PV,
+                        (j > 1 || k > 0) ? 1u : 0u);
+              }
+              if (j - 1 == nt[s] - 1) tc_commit(BAR(B_OFINAL + s));
+            }
+            if (j < nt[s]) {
+              // S_s = Q_s K_j^T
+              tc_fence_after();
+              const uint32_t qbase = sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES;
+              const uint32_t kbase = sbase + SM::KV_OFF + slotK * SM::KV_TILE_BYTES;
+#pragma unroll
+              for (int k = 0; k < D / 16; ++k) {
+                const uint32_t off = (k / 4) * BLK_BYTES + (k % 4) * 32;
+                umma_ss(tmem + S_COL0 + s * 128, make_sdesc(qbase + off, 16, 1024), make_sdesc(kbase + off, 16, 1024),
+                        IDESC_QK, k > 0 ? 1u : 0u);
+              }
+              tc_commit(BAR(B_SFULL + s));
+              if (j == nt[s] - 1) tc_commit(BAR(B_QEMPTY + s));
+            }
+          }
+          if (!ok) break;
+          if (j >= 1) tc_commit(BAR(B_KVEMPTY + slotV));
+          if (j < n_max) tc_commit(BAR(B_KVEMPTY + slotK));
+        }
+        kv_it += 2 * n_max;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue
+    const int s = (warp - 2) >> 2;            // Q tile handled by this warp group
+    const int rb = warp & 3;                  // TMEM lane block this warp may access
+    const int row = rb * 32 + lane;
+    const uint32_t t_s = tmem_addr(tmem, rb * 32, S_COL0 + s * 128);
+    const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
+    uint32_t scnt = 0, ucnt = 0;
+    bool ok = true;
+    for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+      const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+      const int hl = (int)(w % a.head_count);
+      const int nts = __ldg(U + FU_NT_STAGE0 + s);
+      if (nts == 0) continue;
+      const int q_row0 = __ldg(U + FU_Q_ROW0) + s * 128;
+      const int rows_s = min(128, __ldg(U + FU_Q_ROWS) - s * 128);
+      const int q_pos = q_row0 + row;
+      const int nr0 = __ldg(U + FU_NT_RANGE0);
+      const int kvb[2] = {__ldg(U + FU_KV0_BEGIN), __ldg(U + FU_KV1_BEGIN)};
+      const int kve[2] = {__ldg(U + FU_KV0_END), __ldg(U + FU_KV1_END)};
+      const int kvd[2] = {__ldg(U + FU_KV0_DIAG), __ldg(U + FU_KV1_DIAG)};
+      float m_ref = -INFINITY, l = 0.f;
+      for (int j = 0; j < nts && ok; ++j) {
+        const int r = j < nr0 ? 0 : 1;
+        const int ks = r == 0 ? kvb[0] + j * 128 : kvb[1] + (j - nr0) * 128;
+        int limit = kve[r] - ks;                              // valid columns of this tile for this row
+        if (kvd[r]) limit = min(limit, q_pos - ks + 1);
+        ok = mbar_wait_warp(BAR(B_SFULL + s), scnt & 1, wctx, 30 + s);
+        ++scnt;
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sv[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
+        tc_wait_ld();
+        float mx = -INFINITY;
+        if (__any_sync(0xffffffffu, limit < 128)) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float x = c < limit ? __uint_as_float(sv[c]) : -INFINITY;
+            sv[c] = __float_as_uint(x);
+            mx = fmaxf(mx, x);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
+        }
+        mx *= a.scale_log2;
+        // Lazy reference maximum: O and l are only rescaled when the row maximum grew by more than
+        // 2^8, so p <= 256 always and the result is exact up to rounding.
+        const bool grow = mx > m_ref + 8.f;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float m_new = grow ? mx : m_ref;
+          const float f = grow ? ex2(m_ref - m_new) : 1.f;    // m_ref = -inf -> 0
+          l *= f;
+          if (j > 0) {
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t ov[32];
+              tmem_ld32(t_o + c * 32, ov);
+              tc_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+              tmem_st32(t_o + c * 32, ov);
+            }
+          }
+          m_ref = m_new;
+        }
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[c * 32 + 2 * i]), a.scale_log2, -m_ref));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[c * 32 + 2 * i + 1]), a.scale_log2, -m_ref));
+            sum += p0 + p1;
+            pk[i] = pack_bf16(p0, p1);
+          }
+          tmem_st16(t_s + c * 16, pk);
+        }
+        l += sum;
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(BAR(B_PFULL + s));
+      }
+      if (!ok) break;
+      // epilogue: normalised partial output + log-sum-exp
+      ok = mbar_wait_warp(BAR(B_OFINAL + s), ucnt & 1, wctx, 32 + s);
+      ++ucnt;
+      if (!ok) break;
+      tc_fence_after();
+      const float inv_l = 1.f / l;
+      const int64_t prow = (int64_t)__ldg(U + FU_PART_ROW0) + s * 128 + row;
+      float* op = a.o_partial + (prow * a.head_count + hl) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t ov[32];
+        tmem_ld32(t_o + c * 32, ov);
+        tc_wait_ld();
+        if (row < rows_s) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 4) {
+            float4 v4 = make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
+                                    __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
+            *reinterpret_cast<float4*>(op + c * 32 + i) = v4;
+          }
+        }
+      }
+      if (row < rows_s) a.lse_partial[prow * a.head_count + hl] = (m_ref + log2f(l)) * 0.6931471805599453f;
+      tc_fence_before();
+      mbar_arrive(BAR(B_OEMPTY + s));
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  if (*abort_flag) {
+    // A wait gave up: give copies and MMAs still in flight time to land before the CTA's shared
+    // and tensor memory are released.
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+}  // namespace fcp

@@ -1,0 +1,498 @@
+// Device side of libfcp: launchers behind the C ABI, the HBM-bound kernels (LSE merge, backward
+// preprocess, dQ conversion) and the glue around the tensor-core kernels of fcp_fwd.cuh and
+// fcp_bwd.cuh.  No call here allocates device memory except fcp_plan_upload.
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "fcp_bwd.cuh"
+#include "fcp_fwd.cuh"
+
+using namespace fcp;
+
+#define FCP_CUDA_CHECK(expr)                                                             \
+  do {                                                                                   \
+    cudaError_t e_ = (expr);                                                             \
+    if (e_ != cudaSuccess) {                                                             \
+      fcp_set_error("%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e_), __FILE__, __LINE__); \
+      return FCP_ERR_CUDA;                                                               \
+    }                                                                                    \
+  } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Tensor maps
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = (EncodeTiledFn)p;
+  return fn;
+}
+
+// bf16 tensor [T][H][D]; box = 64 columns x 1 head x `box_rows` tokens, 128-byte swizzle, zero fill.
+int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int D, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) {
+    fcp_set_error("cuTensorMapEncodeTiled is not available from the driver");
+    return FCP_ERR_CUDA;
+  }
+  if (((uintptr_t)base & 15) != 0) {
+    fcp_set_error("tensor base %p is not 16-byte aligned", base);
+    return FCP_ERR_INVALID_ARG;
+  }
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
+  const cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    fcp_set_error("cuTensorMapEncodeTiled failed with %d", (int)r);
+    return FCP_ERR_CUDA;
+  }
+  return FCP_OK;
+}
+
+int check_plan(const fcp_plan* plan) {
+  if (!plan) {
+    fcp_set_error("plan is NULL");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if (!plan->d_blob) {
+    fcp_set_error("plan has no device copy: call fcp_plan_upload first");
+    return FCP_ERR_NOT_UPLOADED;
+  }
+  return FCP_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// LSE merge (HBM bound).  One thread owns 8 output columns of one (token, head) row: it reads the
+// row's slot log-sum-exps, forms the exact weights and accumulates 2 x 128-bit loads per slot.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) fcp_merge_kernel(const int32_t* __restrict__ units, const int32_t* __restrict__ slot_offset,
+                                                        const int32_t* __restrict__ slot_rows, const float* __restrict__ o_partial,
+                                                        const float* __restrict__ lse_partial, int head_begin, int head_count,
+                                                        int hq, __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
+  constexpr int TPR = D / 8;                 // threads per (token, head) row
+  constexpr int RPP = 256 / TPR;             // rows per pass
+  const int32_t* U = units + (size_t)blockIdx.x * FCP_MERGE_UNIT_W;
+  const int tok0 = U[MU_TOK_BEGIN], ntok = U[MU_N_TOK], chunk = U[MU_CHUNK], ctok0 = U[MU_CHUNK_TOK_BEGIN];
+  const int s0 = slot_offset[chunk], ns = slot_offset[chunk + 1] - s0;
+  const int sub = threadIdx.x % TPR, rloc = threadIdx.x / TPR;
+  const int n_rows = ntok * head_count;
+  for (int r = rloc; r < n_rows; r += RPP) {
+    const int t = tok0 + r / head_count, hl = r % head_count;
+    const int64_t rel = t - ctok0;
+    float m = -INFINITY;
+    for (int s = 0; s < ns; ++s) m = fmaxf(m, __ldg(lse_partial + ((int64_t)slot_rows[s0 + s] + rel) * head_count + hl));
+    float z = 0.f;
+    for (int s = 0; s < ns; ++s)
+      z += __expf(__ldg(lse_partial + ((int64_t)slot_rows[s0 + s] + rel) * head_count + hl) - m);
+    const float L = m + __logf(z);
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int s = 0; s < ns; ++s) {
+      const int64_t prow = ((int64_t)slot_rows[s0 + s] + rel) * head_count + hl;
+      const float wgt = __expf(__ldg(lse_partial + prow) - L);
+      const float4* src = reinterpret_cast<const float4*>(o_partial + prow * D + sub * 8);
+      const float4 a0 = __ldcs(src), a1 = __ldcs(src + 1);
+      acc[0] += wgt * a0.x; acc[1] += wgt * a0.y; acc[2] += wgt * a0.z; acc[3] += wgt * a0.w;
+      acc[4] += wgt * a1.x; acc[5] += wgt * a1.y; acc[6] += wgt * a1.z; acc[7] += wgt * a1.w;
+    }
+    const int64_t orow = (int64_t)t * hq + head_begin + hl;
+    uint4 pk;
+    pk.x = pack_bf16(acc[0], acc[1]); pk.y = pack_bf16(acc[2], acc[3]);
+    pk.z = pack_bf16(acc[4], acc[5]); pk.w = pack_bf16(acc[6], acc[7]);
+    *reinterpret_cast<uint4*>(o + orow * D + sub * 8) = pk;
+    if (sub == 0) lse[orow] = L;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Backward preprocess (HBM bound): delta[h][t] = sum_c dO[t,h,c] * O[t,h,c], and the forward LSE
+// transposed to [h][t] in log2 units, the layout the backward kernel's per-tile loads want.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256) fcp_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
+                                                        const float* __restrict__ lse, int64_t T, int hq, int64_t t_stride,
+                                                        float* __restrict__ delta_t, float* __restrict__ lse2_t) {
+  constexpr int TPR = D / 8;
+  const int64_t row = ((int64_t)blockIdx.x * 256 + threadIdx.x) / TPR;   // (token, head) row
+  const int sub = threadIdx.x % TPR;
+  float acc = 0.f;
+  if (row < T * hq) {
+    const uint4 a = *reinterpret_cast<const uint4*>(o + row * D + sub * 8);
+    const uint4 b = *reinterpret_cast<const uint4*>(d_o + row * D + sub * 8);
+    const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 fa = __bfloat1622float2(pa[i]), fb = __bfloat1622float2(pb[i]);
+      acc += fa.x * fb.x + fa.y * fb.y;
+    }
+  }
+#pragma unroll
+  for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (row < T * hq && sub == 0) {
+    const int64_t t = row / hq;
+    const int h = (int)(row % hq);
+    delta_t[h * t_stride + t] = acc;
+    lse2_t[h * t_stride + t] = lse[row] * 1.4426950408889634f;
+  }
+}
+
+// fp32 dQ accumulator -> bf16
+__global__ void __launch_bounds__(256) fcp_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq,
+                                                             int64_t n8) {
+  for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n8; i += (int64_t)gridDim.x * 256) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i);
+    const float4 b = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
+    uint4 pk;
+    pk.x = pack_bf16(a.x, a.y); pk.y = pack_bf16(a.z, a.w);
+    pk.z = pack_bf16(b.x, b.y); pk.w = pack_bf16(b.z, b.w);
+    reinterpret_cast<uint4*>(dq)[i] = pk;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Plan upload / destroy / status
+// ---------------------------------------------------------------------------------------------
+extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
+  if (!plan) return FCP_ERR_INVALID_ARG;
+  if (plan->d_blob) return FCP_OK;
+  int dev = 0;
+  FCP_CUDA_CHECK(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  FCP_CUDA_CHECK(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) {
+    fcp_set_error("device %d is sm_%d%d; this library is built for sm_100a only", dev, prop.major, prop.minor);
+    return FCP_ERR_CUDA;
+  }
+  plan->device = dev;
+  plan->sm_count = prop.multiProcessorCount;
+  const std::vector<int32_t>* tabs[6] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges,
+                                         &plan->merge_units, &plan->slot_offset, &plan->slot_rows};
+  size_t off[7];
+  size_t total = 256;  // status words first
+  for (int i = 0; i < 6; ++i) {
+    off[i] = total;
+    total += (tabs[i]->size() * 4 + 255) / 256 * 256;
+  }
+  off[6] = total;
+  void* blob = nullptr;
+  FCP_CUDA_CHECK(cudaMalloc(&blob, total));
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = cudaMemsetAsync(blob, 0, 256, st);
+  for (int i = 0; i < 6 && e == cudaSuccess; ++i)
+    if (!tabs[i]->empty())
+      e = cudaMemcpyAsync((char*)blob + off[i], tabs[i]->data(), tabs[i]->size() * 4, cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) {
+    cudaFree(blob);
+    fcp_set_error("plan upload failed: %s", cudaGetErrorString(e));
+    return FCP_ERR_CUDA;
+  }
+  plan->d_blob = blob;
+  plan->d_status = (int32_t*)blob;
+  plan->d_fwd_units = (int32_t*)((char*)blob + off[0]);
+  plan->d_bwd_units = (int32_t*)((char*)blob + off[1]);
+  plan->d_bwd_qranges = (int32_t*)((char*)blob + off[2]);
+  plan->d_merge_units = (int32_t*)((char*)blob + off[3]);
+  plan->d_slot_offset = (int32_t*)((char*)blob + off[4]);
+  plan->d_slot_rows = (int32_t*)((char*)blob + off[5]);
+  // opt in to the large dynamic shared memory of the tensor-core kernels once
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::DYN_BYTES));
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::DYN_BYTES));
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::DYN_BYTES));
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::DYN_BYTES));
+  return FCP_OK;
+}
+
+extern "C" int fcp_plan_destroy(fcp_plan* plan) {
+  if (!plan) return FCP_OK;
+  if (plan->d_blob) cudaFree(plan->d_blob);
+  delete plan;
+  return FCP_OK;
+}
+
+extern "C" int fcp_last_device_status(const fcp_plan* plan, int32_t* status) {
+  if (!status) return FCP_ERR_INVALID_ARG;
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  FCP_CUDA_CHECK(cudaDeviceSynchronize());
+  FCP_CUDA_CHECK(cudaMemcpy(status, plan->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return FCP_OK;
+}
+
+// scratch layout of fcp_attn_bwd: [dq fp32 accumulator T*hq*D] [delta_t hq*Tpad] [lse2_t hq*Tpad]
+static inline int64_t bwd_tpad(int64_t T) { return (T + 255) / 256 * 256 + 256; }
+
+extern "C" int fcp_plan_workspace_bytes(const fcp_plan* plan, int32_t heads_per_pass, int64_t* o_partial_bytes,
+                                        int64_t* lse_partial_bytes, int64_t* bwd_scratch_bytes) {
+  if (!plan || heads_per_pass <= 0 || heads_per_pass > plan->params.hq) {
+    fcp_set_error("fcp_plan_workspace_bytes: invalid argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  const int64_t D = plan->params.head_dim;
+  if (o_partial_bytes) *o_partial_bytes = plan->R * heads_per_pass * D * 4;
+  if (lse_partial_bytes) *lse_partial_bytes = plan->R * heads_per_pass * 4;
+  if (bwd_scratch_bytes)
+    *bwd_scratch_bytes = plan->T * plan->params.hq * D * 4 + 2 * bwd_tpad(plan->T) * plan->params.hq * 4;
+  return FCP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Compute calls
+// ---------------------------------------------------------------------------------------------
+static int check_heads(const fcp_plan* plan, int head_begin, int head_count) {
+  if (head_begin < 0 || head_count <= 0 || head_begin + head_count > plan->params.hq) {
+    fcp_set_error("head range [%d, %d) outside [0, %d)", head_begin, head_begin + head_count, plan->params.hq);
+    return FCP_ERR_INVALID_ARG;
+  }
+  return FCP_OK;
+}
+
+extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
+                            int32_t head_count, float* o_partial, float* lse_partial, void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!q || !k || !v || !o_partial || !lse_partial) {
+    fcp_set_error("fcp_attn_fwd: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+  const fcp_params& P = plan->params;
+  CUtensorMap tq, tk, tv;
+  if ((rc = make_thd_map(&tq, q, plan->T, P.hq, P.head_dim, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tk, k, plan->T, P.hkv, P.head_dim, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tv, v, plan->T, P.hkv, P.head_dim, 128)) != FCP_OK) return rc;
+  FwdArgs a;
+  a.units = plan->d_fwd_units;
+  a.n_units = (int32_t)(plan->fwd_units.size() / FCP_FWD_UNIT_W);
+  a.head_begin = head_begin;
+  a.head_count = head_count;
+  a.hq = P.hq;
+  a.hkv = P.hkv;
+  a.scale_log2 = P.scale * 1.4426950408889634f;
+  a.o_partial = o_partial;
+  a.lse_partial = lse_partial;
+  a.status = plan->d_status;
+  const int64_t n_work = (int64_t)a.n_units * head_count;
+  const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
+  if (grid == 0) return FCP_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (P.head_dim == 128)
+    fcp_fwd_kernel<128><<<grid, FWD_THREADS, FwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, a);
+  else
+    fcp_fwd_kernel<64><<<grid, FWD_THREADS, FwdSmem<64>::DYN_BYTES, st>>>(tq, tk, tv, a);
+  FCP_CUDA_CHECK(cudaGetLastError());
+  return FCP_OK;
+}
+
+extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
+                             int32_t head_begin, int32_t head_count, void* o, float* lse, void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!o_partial || !lse_partial || !o || !lse) {
+    fcp_set_error("fcp_lse_merge: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+  const fcp_params& P = plan->params;
+  const int n_units = (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W);
+  if (n_units == 0) return FCP_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (P.head_dim == 128)
+    fcp_merge_kernel<128><<<n_units, 256, 0, st>>>(plan->d_merge_units, plan->d_slot_offset, plan->d_slot_rows, o_partial,
+                                                   lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, lse);
+  else
+    fcp_merge_kernel<64><<<n_units, 256, 0, st>>>(plan->d_merge_units, plan->d_slot_offset, plan->d_slot_rows, o_partial,
+                                                  lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, lse);
+  FCP_CUDA_CHECK(cudaGetLastError());
+  return FCP_OK;
+}
+
+extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                            const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* scratch,
+                            int64_t scratch_bytes, void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv || !scratch) {
+    fcp_set_error("fcp_attn_bwd: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  const fcp_params& P = plan->params;
+  const int64_t T = plan->T, D = P.head_dim;
+  int64_t need = 0;
+  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &need);
+  if (scratch_bytes < need) {
+    fcp_set_error("fcp_attn_bwd: scratch of %lld bytes, %lld needed", (long long)scratch_bytes, (long long)need);
+    return FCP_ERR_WORKSPACE;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t tpad = bwd_tpad(T);
+  float* dq_acc = (float*)scratch;
+  float* delta_t = dq_acc + T * P.hq * D;
+  float* lse2_t = delta_t + tpad * P.hq;
+  FCP_CUDA_CHECK(cudaMemsetAsync(scratch, 0, (size_t)need, st));
+  {
+    const int64_t rows = T * P.hq;
+    const int tpr = (int)D / 8;
+    const int64_t blocks = (rows * tpr + 255) / 256;
+    if (D == 128)
+      fcp_delta_kernel<128><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
+                                                              tpad, delta_t, lse2_t);
+    else
+      fcp_delta_kernel<64><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
+                                                             tpad, delta_t, lse2_t);
+    FCP_CUDA_CHECK(cudaGetLastError());
+  }
+  CUtensorMap tq, tk, tv, tdo;
+  if ((rc = make_thd_map(&tq, q, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tk, k, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tv, v, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tdo, d_o, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
+  BwdArgs a;
+  a.units = plan->d_bwd_units;
+  a.qranges = plan->d_bwd_qranges;
+  a.n_units = (int32_t)(plan->bwd_units.size() / FCP_BWD_UNIT_W);
+  a.hq = P.hq;
+  a.hkv = P.hkv;
+  a.T = T;
+  a.t_stride = tpad;
+  a.scale = P.scale;
+  a.scale_log2 = P.scale * 1.4426950408889634f;
+  a.delta_t = delta_t;
+  a.lse2_t = lse2_t;
+  a.dq_acc = dq_acc;
+  a.dk = (__nv_bfloat16*)dk;
+  a.dv = (__nv_bfloat16*)dv;
+  a.status = plan->d_status;
+  const int64_t n_work = (int64_t)a.n_units * P.hkv;
+  const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
+  if (grid > 0) {
+    if (D == 128)
+      fcp_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
+    else
+      fcp_bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
+    FCP_CUDA_CHECK(cudaGetLastError());
+  }
+  {
+    const int64_t n8 = T * P.hq * D / 8;
+    const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)plan->sm_count * 16);
+    fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8);
+    FCP_CUDA_CHECK(cudaGetLastError());
+  }
+  return FCP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Whole path from host buffers
+// ---------------------------------------------------------------------------------------------
+namespace {
+struct HostLayout {
+  int64_t q, k, v, d_o, o, lse, dq, dk, dv, scratch, o_part, lse_part, total;
+  int heads_per_pass;
+};
+inline int64_t al(int64_t x) { return (x + 255) / 256 * 256; }
+
+HostLayout host_layout(const fcp_plan* plan, int64_t limit_bytes) {
+  const fcp_params& P = plan->params;
+  const int64_t T = plan->T, D = P.head_dim;
+  HostLayout L{};
+  int64_t off = 0;
+  auto take = [&](int64_t bytes) { int64_t o = off; off += al(bytes); return o; };
+  L.q = take(T * P.hq * D * 2);
+  L.k = take(T * P.hkv * D * 2);
+  L.v = take(T * P.hkv * D * 2);
+  L.d_o = take(T * P.hq * D * 2);
+  L.o = take(T * P.hq * D * 2);
+  L.lse = take(T * P.hq * 4);
+  L.dq = take(T * P.hq * D * 2);
+  L.dk = take(T * P.hkv * D * 2);
+  L.dv = take(T * P.hkv * D * 2);
+  int64_t scratch = 0;
+  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
+  // the partial buffers are dead once merged, so they share memory with the backward scratch
+  const int64_t per_head = al(plan->R * D * 4) + al(plan->R * 4);
+  int hpp = P.hq;
+  if (limit_bytes > 0)
+    while (hpp > 1 && off + std::max<int64_t>(scratch, per_head * hpp) > limit_bytes) --hpp;
+  L.heads_per_pass = hpp;
+  L.scratch = off;
+  L.o_part = off;
+  L.lse_part = off + al(plan->R * hpp * D * 4);
+  off += al(std::max<int64_t>(scratch, al(plan->R * hpp * D * 4) + al(plan->R * hpp * 4)));
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+extern "C" int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes) {
+  if (!plan || !bytes) return FCP_ERR_INVALID_ARG;
+  // smallest useful workspace: one head per pass would always fit, but prefer all heads when the
+  // partial buffers stay below 48 GiB
+  HostLayout L = host_layout(plan, 0);
+  if (L.total > (int64_t(96) << 30)) L = host_layout(plan, int64_t(96) << 30);
+  *bytes = L.total;
+  return FCP_OK;
+}
+
+extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host, const void* v_host,
+                                     const void* d_o_host, void* o_host, float* lse_host, void* dq_host, void* dk_host,
+                                     void* dv_host, void* workspace, int64_t workspace_bytes, void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !lse_host || !dq_host || !dk_host || !dv_host ||
+      !workspace) {
+    fcp_set_error("fcp_attn_fwd_bwd_host: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  const HostLayout L = host_layout(plan, workspace_bytes);
+  if (L.total > workspace_bytes) {
+    fcp_set_error("fcp_attn_fwd_bwd_host: workspace of %lld bytes, %lld needed", (long long)workspace_bytes,
+                  (long long)L.total);
+    return FCP_ERR_WORKSPACE;
+  }
+  const fcp_params& P = plan->params;
+  const int64_t T = plan->T, D = P.head_dim;
+  char* w = (char*)workspace;
+  cudaStream_t st = (cudaStream_t)stream;
+  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q, q_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k, k_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v, v_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o, d_o_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, st));
+  for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
+    const int hc = std::min(L.heads_per_pass, P.hq - h0);
+    if ((rc = fcp_attn_fwd(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part), st)) != FCP_OK)
+      return rc;
+    if ((rc = fcp_lse_merge(plan, (float*)(w + L.o_part), (float*)(w + L.lse_part), h0, hc, w + L.o, (float*)(w + L.lse), st)) != FCP_OK)
+      return rc;
+  }
+  int64_t scratch = 0;
+  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
+  if ((rc = fcp_attn_bwd(plan, w + L.q, w + L.k, w + L.v, w + L.o, w + L.d_o, (float*)(w + L.lse), w + L.dq, w + L.dk,
+                         w + L.dv, w + L.scratch, scratch, st)) != FCP_OK)
+    return rc;
+  FCP_CUDA_CHECK(cudaMemcpyAsync(o_host, w + L.o, T * P.hq * D * 2, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(lse_host, w + L.lse, T * P.hq * 4, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(dq_host, w + L.dq, T * P.hq * D * 2, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(dk_host, w + L.dk, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(dv_host, w + L.dv, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaStreamSynchronize(st));
+  return FCP_OK;
+}

@@ -1,0 +1,435 @@
+// Host side of libfcp: the strategy planner (Sec. 4.4, Eq. 7, Algorithm 1) and the block plan that
+// the kernels consume.  Plain C++, integers and doubles only; nothing here touches the GPU.
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <limits>
+#include <numeric>
+#include <vector>
+
+#include "fcp_plan.hpp"
+
+namespace {
+thread_local char g_err[512] = "";
+}
+
+void fcp_set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+extern "C" const char* fcp_last_error_message(void) { return g_err; }
+
+extern "C" const char* fcp_status_string(int status) {
+  switch (status) {
+    case FCP_OK: return "FCP_OK";
+    case FCP_ERR_INVALID_ARG: return "FCP_ERR_INVALID_ARG";
+    case FCP_ERR_INFEASIBLE: return "FCP_ERR_INFEASIBLE";
+    case FCP_ERR_UNSUPPORTED: return "FCP_ERR_UNSUPPORTED";
+    case FCP_ERR_WORKSPACE: return "FCP_ERR_WORKSPACE";
+    case FCP_ERR_CUDA: return "FCP_ERR_CUDA";
+    case FCP_ERR_TIMEOUT: return "FCP_ERR_TIMEOUT";
+    case FCP_ERR_NOT_UPLOADED: return "FCP_ERR_NOT_UPLOADED";
+    default: return "FCP_ERR_UNKNOWN";
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Strategy planner
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct GroupSums {  // sums over the sequences of one atomic group
+  double quad = 0.0, lin = 0.0, tot = 0.0;
+};
+
+// T(G, d), Eq. 6: T_cp + T_cm - min(T_cpa, T_cma).  Eqs. 4-5 are written per group; the d ranks of
+// a group share the compute terms, and ring communication only exists for d > 1.
+double group_time(const GroupSums& g, int d, const fcp_cost_coeffs& c) {
+  const double t_cpa = g.quad / d;
+  const double t_cp = (g.quad + g.lin) / d + c.beta1;
+  const double t_cm = d > 1 ? (c.alpha3 * g.tot) / c.v + c.beta2 : 0.0;
+  const double t_cma = t_cm;
+  return t_cp + t_cm - std::min(t_cpa, t_cma);
+}
+
+}  // namespace
+
+extern "C" int fcp_plan_strategy(const int32_t* seqlens, int32_t B, int32_t N, double E,
+                                 double M_token, double M_ms, const fcp_cost_coeffs* coeffs,
+                                 int32_t* group_of, int32_t* cp_degree, int32_t* n_groups,
+                                 double* makespan) {
+  if (!seqlens || !coeffs || B <= 0 || N <= 0 || !(E > M_ms) || !(M_token > 0.0) || !(coeffs->v > 0.0)) {
+    fcp_set_error("fcp_plan_strategy: invalid argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if (N > FCP_MAX_DEGREE) {
+    fcp_set_error("fcp_plan_strategy: N=%d exceeds FCP_MAX_DEGREE=%d", N, FCP_MAX_DEGREE);
+    return FCP_ERR_UNSUPPORTED;
+  }
+  for (int i = 0; i < B; ++i)
+    if (seqlens[i] <= 0) {
+      fcp_set_error("fcp_plan_strategy: seqlens[%d]=%d", i, seqlens[i]);
+      return FCP_ERR_INVALID_ARG;
+    }
+
+  // Stage 1: best-fit-decreasing.  Longest first (ties: lower index); a sequence goes to the open
+  // group with the least remaining headroom that still holds it (ties: lowest group), otherwise it
+  // opens a group of d_min = ceil(need / budget) ranks.
+  const double budget = E - M_ms;
+  std::vector<int> order(B);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return seqlens[a] > seqlens[b]; });
+  std::vector<double> headroom;
+  std::vector<int> dmin;
+  std::vector<int> gof(B, 0);
+  for (int i : order) {
+    const double need = double(seqlens[i]) * M_token;
+    int best = -1;
+    for (int g = 0; g < (int)headroom.size(); ++g)
+      if (headroom[g] >= need && (best < 0 || headroom[g] < headroom[best])) best = g;
+    if (best < 0) {
+      const int dm = std::max(1, (int)std::ceil(need / budget));
+      headroom.push_back(dm * budget - need);
+      dmin.push_back(dm);
+      best = (int)headroom.size() - 1;
+    } else {
+      headroom[best] -= need;
+    }
+    gof[i] = best;
+  }
+  const int K = (int)dmin.size();
+  long long need_ranks = 0;
+  for (int d : dmin) need_ranks += d;
+  if (need_ranks > N) {
+    fcp_set_error("fcp_plan_strategy: minimum degrees need %lld ranks, only %d available", need_ranks, N);
+    return FCP_ERR_INFEASIBLE;
+  }
+
+  // Per-group sums in sequence-index order.
+  std::vector<GroupSums> sums(K);
+  for (int i = 0; i < B; ++i) {
+    const double L = double(seqlens[i]);
+    const double eta = coeffs->eta ? coeffs->eta[i] : 0.0;
+    GroupSums& g = sums[gof[i]];
+    g.quad += coeffs->alpha1 * (1.0 + eta) * L * L;
+    g.lin += coeffs->alpha2 * L;
+    g.tot += L;
+  }
+
+  // Stage 2: Algorithm 1.  Only DP[0][0] is finite initially; strict '<' keeps the smallest d on ties.
+  const double INF = std::numeric_limits<double>::infinity();
+  std::vector<double> dp((size_t)(K + 1) * (N + 1), INF);
+  std::vector<int> path((size_t)(K + 1) * (N + 1), 0);
+  auto at = [&](int k, int j) -> size_t { return (size_t)k * (N + 1) + j; };
+  dp[at(0, 0)] = 0.0;
+  int before = 0;                       // sum of d_min of groups 1..k-1
+  int remain = (int)need_ranks;         // sum of d_min of groups k+1..K'
+  for (int k = 1; k <= K; ++k) {
+    remain -= dmin[k - 1];
+    for (int j = before + dmin[k - 1]; j <= N - remain; ++j) {
+      for (int d = dmin[k - 1]; d <= j - before; ++d) {
+        const double cost = std::max(dp[at(k - 1, j - d)], group_time(sums[k - 1], d, *coeffs));
+        if (cost < dp[at(k, j)]) {
+          dp[at(k, j)] = cost;
+          path[at(k, j)] = d;
+        }
+      }
+    }
+    before += dmin[k - 1];
+  }
+  std::vector<int> deg(K, 0);
+  for (int p = K, q = N; p > 0; --p) {
+    deg[p - 1] = path[at(p, q)];
+    q -= deg[p - 1];
+  }
+  for (int i = 0; i < B; ++i) {
+    if (group_of) group_of[i] = gof[i];
+    if (cp_degree) cp_degree[i] = deg[gof[i]];
+  }
+  if (n_groups) *n_groups = K;
+  if (makespan) *makespan = dp[at(K, N)];
+  return FCP_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Block plan
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+struct Pair {
+  int32_t seq, rank, step, qc, kc, kind;
+  bool operator<(const Pair& o) const {
+    if (rank != o.rank) return rank < o.rank;
+    if (step != o.step) return step < o.step;
+    if (qc != o.qc) return qc < o.qc;
+    return kc < o.kc;
+  }
+};
+
+inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+}  // namespace
+
+extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
+                               const fcp_params* params, fcp_plan** out) {
+  if (!seqlens || !cp_degrees || !params || !out || B <= 0) {
+    fcp_set_error("fcp_plan_blocks: invalid argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  *out = nullptr;
+  if ((params->head_dim != 64 && params->head_dim != 128) || params->hq <= 0 || params->hkv <= 0 ||
+      params->hq % params->hkv != 0) {
+    fcp_set_error("fcp_plan_blocks: unsupported shape hq=%d hkv=%d head_dim=%d", params->hq, params->hkv,
+                  params->head_dim);
+    return FCP_ERR_UNSUPPORTED;
+  }
+  int64_t T = 0;
+  for (int b = 0; b < B; ++b) {
+    if (seqlens[b] <= 0 || cp_degrees[b] <= 0) {
+      fcp_set_error("fcp_plan_blocks: sequence %d has length %d, degree %d", b, seqlens[b], cp_degrees[b]);
+      return FCP_ERR_INVALID_ARG;
+    }
+    if (cp_degrees[b] > FCP_MAX_DEGREE) {
+      fcp_set_error("fcp_plan_blocks: degree %d > FCP_MAX_DEGREE", cp_degrees[b]);
+      return FCP_ERR_UNSUPPORTED;
+    }
+    T += seqlens[b];
+  }
+  if (T >= (int64_t(1) << 31) - 2 * FCP_FWD_UNIT_ROWS) {
+    fcp_set_error("fcp_plan_blocks: %lld tokens exceed the 2^31 limit", (long long)T);
+    return FCP_ERR_INVALID_ARG;
+  }
+
+  fcp_plan* p = new fcp_plan();
+  p->params = *params;
+  if (!(p->params.scale > 0.f)) p->params.scale = 1.0f / std::sqrt((float)params->head_dim);
+  p->B = B;
+  p->T = T;
+  p->cu_seqlens.assign(B + 1, 0);
+  for (int b = 0; b < B; ++b) p->cu_seqlens[b + 1] = p->cu_seqlens[b] + seqlens[b];
+
+  // Chunk bounds and pairs.
+  p->chunk_offset.push_back(0);
+  std::vector<Pair> pairs;
+  for (int b = 0; b < B; ++b) {
+    const int64_t L = seqlens[b];
+    const int d = cp_degrees[b];
+    const int32_t t0 = p->cu_seqlens[b];
+    const size_t base = p->chunk_bounds.size();
+    for (int c = 0; c <= 2 * d; ++c) p->chunk_bounds.push_back(t0 + (int32_t)((int64_t)c * L / (2 * d)));
+    p->chunk_offset.push_back((int32_t)p->chunk_bounds.size());
+    auto nonempty = [&](int c) { return p->chunk_bounds[base + c + 1] > p->chunk_bounds[base + c]; };
+    std::vector<Pair> sp;
+    auto add = [&](int r, int s, int qc, int kc) {
+      if (nonempty(qc) && nonempty(kc)) sp.push_back(Pair{b, r, s, qc, kc, qc == kc ? 1 : 0});
+    };
+    const int last = 2 * d - 1;
+    for (int r = 0; r < d; ++r)
+      for (int s = 0; s < d; ++s) {
+        const int j = ((r - s) % d + d) % d;   // rank whose K/V visits at this ring step
+        if (s == 0) {
+          add(r, s, r, r);
+          add(r, s, last - r, r);
+          add(r, s, last - r, last - r);
+        } else if (j < r) {
+          add(r, s, r, j);
+          add(r, s, last - r, j);
+        } else {
+          add(r, s, last - r, j);
+          add(r, s, last - r, last - j);
+        }
+      }
+    std::sort(sp.begin(), sp.end());
+    pairs.insert(pairs.end(), sp.begin(), sp.end());
+  }
+  for (const Pair& x : pairs) {
+    const int32_t row[6] = {x.seq, x.rank, x.step, x.qc, x.kc, x.kind};
+    p->pairs.insert(p->pairs.end(), row, row + 6);
+  }
+
+  // Items: one per (seq, rank, step, q_chunk); slot = order of the step among the steps touching
+  // that Q chunk; partial rows are laid out in item order.
+  const int n_chunks_total = p->chunk_offset[B] - B;  // sum of 2d
+  std::vector<int32_t> chunk_index0(B + 1, 0);        // global chunk index of chunk 0 of each sequence
+  for (int b = 0; b < B; ++b) chunk_index0[b + 1] = chunk_index0[b] + 2 * cp_degrees[b];
+  std::vector<std::vector<std::pair<int, int>>> chunk_items(n_chunks_total);  // (step, item index)
+  int64_t row = 0;
+  for (size_t i = 0; i < pairs.size();) {
+    size_t n = 1;
+    while (i + n < pairs.size() && pairs[i + n].seq == pairs[i].seq && pairs[i + n].rank == pairs[i].rank &&
+           pairs[i + n].step == pairs[i].step && pairs[i + n].qc == pairs[i].qc)
+      ++n;
+    const Pair& x = pairs[i];
+    const int item = (int)(p->items.size() / 8);
+    const int32_t cb = p->chunk_offset[x.seq] + x.qc;
+    const int32_t len = p->chunk_bounds[cb + 1] - p->chunk_bounds[cb];
+    const int32_t rowv[8] = {x.seq, x.rank, x.step, x.qc, 0, (int32_t)row, (int32_t)n, (int32_t)i};
+    p->items.insert(p->items.end(), rowv, rowv + 8);
+    chunk_items[chunk_index0[x.seq] + x.qc].push_back({x.step, item});
+    row += len;
+    if (row >= (int64_t(1) << 31) - 2 * FCP_FWD_UNIT_ROWS) {
+      delete p;
+      fcp_set_error("fcp_plan_blocks: partial rows exceed the 2^31 limit");
+      return FCP_ERR_INVALID_ARG;
+    }
+    i += n;
+  }
+  p->R = row;
+  p->slot_offset.push_back(0);
+  for (int c = 0; c < n_chunks_total; ++c) {
+    auto& v = chunk_items[c];
+    std::sort(v.begin(), v.end());
+    for (size_t k = 0; k < v.size(); ++k) {
+      p->items[(size_t)v[k].second * 8 + 4] = (int32_t)k;
+      p->slot_rows.push_back(p->items[(size_t)v[k].second * 8 + 5]);
+    }
+    p->slot_offset.push_back((int32_t)p->slot_rows.size());
+  }
+
+  // ---- derived work lists (execution order; not part of the canonical tables) ----
+  // Forward: an item's Q chunk is cut into units of two adjacent 128-row tiles.  KV ranges of an
+  // item are its pairs in kv_chunk order, so a DIAG range (kv_chunk == q_chunk) is always last.
+  struct FU { int32_t f[FCP_FWD_UNIT_W]; };
+  std::vector<FU> fus;
+  const int n_items = (int)(p->items.size() / 8);
+  for (int it = 0; it < n_items; ++it) {
+    const int32_t* I = &p->items[(size_t)it * 8];
+    const int b = I[0], qc = I[3], np = I[6], fp = I[7];
+    const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+    const int32_t q0 = cbp[qc], q1 = cbp[qc + 1];
+    int32_t kb[2] = {0, 0}, ke[2] = {0, 0}, kd[2] = {0, 0};
+    for (int r = 0; r < np; ++r) {
+      const Pair& x = pairs[fp + r];
+      kb[r] = cbp[x.kc];
+      ke[r] = cbp[x.kc + 1];
+      kd[r] = x.kind;
+    }
+    const int last = np - 1;
+    const int nt_first = np == 2 ? ceil_div(ke[0] - kb[0], FCP_TILE) : 0;
+    for (int32_t off = 0; off < q1 - q0; off += FCP_FWD_UNIT_ROWS) {
+      FU u{};
+      const int32_t rows = std::min<int32_t>(FCP_FWD_UNIT_ROWS, q1 - q0 - off);
+      u.f[FU_Q_ROW0] = q0 + off;
+      u.f[FU_Q_ROWS] = rows;
+      u.f[FU_PART_ROW0] = I[5] + off;
+      u.f[FU_N_RANGES] = np;
+      u.f[FU_KV0_BEGIN] = kb[0]; u.f[FU_KV0_END] = ke[0]; u.f[FU_KV0_DIAG] = kd[0];
+      u.f[FU_KV1_BEGIN] = kb[1]; u.f[FU_KV1_END] = ke[1]; u.f[FU_KV1_DIAG] = kd[1];
+      for (int s = 0; s < 2; ++s) {
+        const int32_t rs = std::min<int32_t>(FCP_TILE, rows - s * FCP_TILE);
+        int nt = 0;
+        if (rs > 0) {
+          if (kd[last]) nt = ceil_div((int64_t)off + s * FCP_TILE + rs, FCP_TILE);  // keys up to the last row
+          else nt = ceil_div(ke[last] - kb[last], FCP_TILE);
+          nt += nt_first;
+        }
+        u.f[FU_NT_STAGE0 + s] = nt;
+      }
+      u.f[FU_NT_RANGE0] = np == 2 ? nt_first : 0x7fffffff;
+      u.f[FU_ITEM] = it;
+      fus.push_back(u);
+    }
+  }
+  std::stable_sort(fus.begin(), fus.end(), [](const FU& a, const FU& b) {
+    return a.f[FU_NT_STAGE0] + a.f[FU_NT_STAGE1] > b.f[FU_NT_STAGE0] + b.f[FU_NT_STAGE1];
+  });
+  p->fwd_units.reserve(fus.size() * FCP_FWD_UNIT_W);
+  for (const FU& u : fus) p->fwd_units.insert(p->fwd_units.end(), u.f, u.f + FCP_FWD_UNIT_W);
+
+  // Backward: one unit per 128-key tile of every KV chunk; it visits the Q chunks of all block
+  // pairs whose kv_chunk is this chunk (q_chunk >= kv_chunk), the DIAG pair from its own tile on.
+  struct BU { int32_t f[FCP_BWD_UNIT_W]; };
+  std::vector<BU> bus;
+  {
+    // pairs grouped by (seq, kv_chunk), Q chunks ascending
+    std::vector<std::vector<std::pair<int, int>>> by_kv(n_chunks_total);  // (q_chunk, kind)
+    for (const Pair& x : pairs) by_kv[chunk_index0[x.seq] + x.kc].push_back({x.qc, x.kind});
+    for (int b = 0; b < B; ++b) {
+      const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+      for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
+        auto& v = by_kv[chunk_index0[b] + c];
+        if (v.empty()) continue;
+        std::sort(v.begin(), v.end());
+        const int32_t first = (int32_t)(p->bwd_qranges.size() / FCP_BWD_QRANGE_W);
+        for (auto& qk : v) {
+          const int32_t rowq[4] = {cbp[qk.first], cbp[qk.first + 1], qk.second, 0};
+          p->bwd_qranges.insert(p->bwd_qranges.end(), rowq, rowq + 4);
+        }
+        const int32_t k0 = cbp[c], k1 = cbp[c + 1];
+        for (int32_t off = 0, t = 0; off < k1 - k0; off += FCP_TILE, ++t) {
+          BU u{};
+          u.f[BU_KV_ROW0] = k0 + off;
+          u.f[BU_KV_ROWS] = std::min<int32_t>(FCP_TILE, k1 - k0 - off);
+          u.f[BU_FIRST_QRANGE] = first;
+          u.f[BU_N_QRANGES] = (int32_t)v.size();
+          u.f[BU_KV_TILE] = t;
+          int cost = 0;
+          for (auto& qk : v) {
+            const int nt = ceil_div(cbp[qk.first + 1] - cbp[qk.first], FCP_TILE);
+            cost += qk.second ? nt - t : nt;
+          }
+          u.f[BU_COST] = cost;
+          u.f[BU_SEQ] = b;
+          bus.push_back(u);
+        }
+      }
+    }
+  }
+  std::stable_sort(bus.begin(), bus.end(), [](const BU& a, const BU& b) { return a.f[BU_COST] > b.f[BU_COST]; });
+  for (const BU& u : bus) p->bwd_units.insert(p->bwd_units.end(), u.f, u.f + FCP_BWD_UNIT_W);
+
+  // Merge: runs of up to FCP_MERGE_TOKENS tokens inside one chunk.
+  for (int b = 0; b < B; ++b) {
+    const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+    for (int c = 0; c < 2 * cp_degrees[b]; ++c)
+      for (int32_t t = cbp[c]; t < cbp[c + 1]; t += FCP_MERGE_TOKENS) {
+        const int32_t rowm[4] = {t, std::min<int32_t>(FCP_MERGE_TOKENS, cbp[c + 1] - t), chunk_index0[b] + c, cbp[c]};
+        p->merge_units.insert(p->merge_units.end(), rowm, rowm + 4);
+      }
+  }
+  *out = p;
+  return FCP_OK;
+}
+
+extern "C" int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count) {
+  if (!plan || !host_ptr || !count) return FCP_ERR_INVALID_ARG;
+  const std::vector<int32_t>* v = nullptr;
+  switch (which) {
+    case FCP_TABLE_CU_SEQLENS: v = &plan->cu_seqlens; break;
+    case FCP_TABLE_CHUNK_OFFSET: v = &plan->chunk_offset; break;
+    case FCP_TABLE_CHUNK_BOUNDS: v = &plan->chunk_bounds; break;
+    case FCP_TABLE_PAIRS: v = &plan->pairs; break;
+    case FCP_TABLE_ITEMS: v = &plan->items; break;
+    case FCP_TABLE_SLOT_OFFSET: v = &plan->slot_offset; break;
+    case FCP_TABLE_SLOT_ROWS: v = &plan->slot_rows; break;
+    case FCP_TABLE_FWD_UNITS: v = &plan->fwd_units; break;
+    case FCP_TABLE_BWD_UNITS: v = &plan->bwd_units; break;
+    case FCP_TABLE_BWD_QRANGES: v = &plan->bwd_qranges; break;
+    case FCP_TABLE_MERGE_UNITS: v = &plan->merge_units; break;
+    default: fcp_set_error("fcp_plan_get: unknown table %d", which); return FCP_ERR_INVALID_ARG;
+  }
+  *host_ptr = v->data();
+  *count = (int64_t)v->size();
+  return FCP_OK;
+}
+
+extern "C" int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value) {
+  if (!plan || !value) return FCP_ERR_INVALID_ARG;
+  switch (which) {
+    case 0: *value = plan->T; break;
+    case 1: *value = plan->R; break;
+    case 2: *value = (int64_t)plan->pairs.size() / 6; break;
+    case 3: *value = (int64_t)plan->items.size() / 8; break;
+    case 4: *value = (int64_t)plan->fwd_units.size() / FCP_FWD_UNIT_W; break;
+    case 5: *value = (int64_t)plan->bwd_units.size() / FCP_BWD_UNIT_W; break;
+    case 6: *value = (int64_t)plan->merge_units.size() / FCP_MERGE_UNIT_W; break;
+    case 7: *value = plan->B; break;
+    default: return FCP_ERR_INVALID_ARG;
+  }
+  return FCP_OK;
+}

@@ -1,0 +1,76 @@
+"""Device-buffer plumbing around the C ABI for tests, the smoke check and the benchmark: allocates
+torch tensors, calls the library, returns numpy results.  No arithmetic of the method happens here."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import fcp, synth
+
+
+def to_dev_bf16(bits: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+
+def bf16_dev_to_f64(t: torch.Tensor) -> np.ndarray:
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+class DeviceState:
+    """All device buffers of one workload (inputs, partials, outputs, scratch) and its uploaded plan."""
+
+    def __init__(self, w: synth.Workload, q, k, v, do=None, heads_per_pass=None):
+        self.w = w
+        self.plan = fcp.fcp_plan_blocks(w.seqlens, w.cp_degrees, w.hq, w.hkv, w.head_dim).upload()
+        T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
+        self.hpp = heads_per_pass or hq
+        self.q, self.k, self.v = to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v)
+        self.do = to_dev_bf16(do) if do is not None else None
+        R = self.plan.info("R")
+        self.R = R
+        self.o_part = torch.empty((R, self.hpp, D), dtype=torch.float32, device="cuda")
+        self.lse_part = torch.empty((R, self.hpp), dtype=torch.float32, device="cuda")
+        self.o = torch.empty((T, hq, D), dtype=torch.bfloat16, device="cuda")
+        self.lse = torch.empty((T, hq), dtype=torch.float32, device="cuda")
+        if do is not None:
+            self.dq = torch.empty((T, hq, D), dtype=torch.bfloat16, device="cuda")
+            self.dk = torch.empty((T, hkv, D), dtype=torch.bfloat16, device="cuda")
+            self.dv = torch.empty((T, hkv, D), dtype=torch.bfloat16, device="cuda")
+            self.scratch_bytes = self.plan.workspace_bytes(1)[2]
+            self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device="cuda")
+
+    def forward(self, stream=None):
+        st = (stream or torch.cuda.current_stream()).cuda_stream
+        for h0 in range(0, self.w.hq, self.hpp):
+            hc = min(self.hpp, self.w.hq - h0)
+            fcp.fcp_attn_fwd(self.plan, self.q, self.k, self.v, self.o_part, self.lse_part, h0, hc, st)
+            fcp.fcp_lse_merge(self.plan, self.o_part, self.lse_part, self.o, self.lse, h0, hc, st)
+
+    def backward(self, stream=None):
+        st = (stream or torch.cuda.current_stream()).cuda_stream
+        fcp.fcp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
+                         self.scratch, self.scratch_bytes, st)
+
+    def check_status(self):
+        st = self.plan.device_status()
+        if st[0] != 0:
+            raise RuntimeError(f"device status {fcp.status_string(int(st[0]))}: where={st[1]} block={st[2]} thread={st[3]}")
+
+
+def run_fwd_bwd(w, q, k, v, do=None, heads_per_pass=None, keep_partials=False):
+    ds = DeviceState(w, q, k, v, do, heads_per_pass)
+    ds.forward()
+    out = {}
+    if do is not None:
+        ds.backward()
+    torch.cuda.synchronize()
+    ds.check_status()
+    out["o"] = bf16_dev_to_f64(ds.o)
+    out["lse"] = ds.lse.cpu().numpy().astype(np.float64)
+    if keep_partials:
+        out["o_partial"] = ds.o_part.cpu().numpy()
+        out["lse_partial"] = ds.lse_part.cpu().numpy()
+    if do is not None:
+        out["dq"], out["dk"], out["dv"] = bf16_dev_to_f64(ds.dq), bf16_dev_to_f64(ds.dk), bf16_dev_to_f64(ds.dv)
+    out["state"] = ds
+    return out
