@@ -141,10 +141,13 @@ int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void*
  *     LSE = m + log sum_s exp(lse_s - m),  o = sum_s exp(lse_s - LSE) * o_s     (m = max_s lse_s)
  * (the re-association of the softmax sum implied by ring-style CP, Sec. 3.2).
  * Writes o[T][hq][D] bf16 and lse[T][hq] fp32 for heads [head_begin, head_begin+head_count); the
- * partial buffers have head_count heads (the layout fcp_attn_fwd wrote).
+ * partial buffers have head_count heads (the layout fcp_attn_fwd wrote).  o_f32 is optional
+ * (NULL to skip): the same output [T][hq][D] before the rounding to bf16, for callers that keep an
+ * fp32 activation stream.
  */
 int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
-                  int32_t head_begin, int32_t head_count, void* o, float* lse, void* stream);
+                  int32_t head_begin, int32_t head_count, void* o, float* o_f32, float* lse,
+                  void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * fcp_attn_bwd — device.  Gradients of Eq. 1 with the causal mask, evaluated over the plan's
@@ -174,6 +177,16 @@ int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* 
 /* Device-side status word of the last kernels run with this plan (0 = fine; FCP_ERR_TIMEOUT if a
  * bounded wait inside a kernel expired).  Synchronises the device.                               */
 int fcp_last_device_status(const fcp_plan* plan, int32_t* status);
+
+/* Kernel timing for benchmarks.  fcp_plan_set_profiling(plan, 1) makes every compute call record a
+ * CUDA event pair around each of its kernels on the launching stream (a ring of the last 64 launches
+ * per kind); fcp_plan_kernel_ms returns, after the caller has synchronised, the number of recorded
+ * launches of `kind` and their mean duration in milliseconds.  kind: 0 forward attention,
+ * 1 LSE merge, 2 backward preprocess (accumulator clear + delta), 3 backward attention,
+ * 4 dQ conversion.  fcp_plan_set_profiling(plan, 0) stops recording and clears the ring.        */
+#define FCP_KERNEL_KINDS 5
+int fcp_plan_set_profiling(fcp_plan* plan, int32_t enable);
+int fcp_plan_kernel_ms(const fcp_plan* plan, int32_t kind, int32_t* launches, float* mean_ms);
 
 const char* fcp_status_string(int status);
 const char* fcp_last_error_message(void);

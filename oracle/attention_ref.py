@@ -47,7 +47,7 @@ import numpy as np
 
 __all__ = [
     "attention_fwd_seq", "attention_bwd_seq", "attention_fwd_packed", "attention_bwd_packed",
-    "attention_row", "partial_attention", "merge_partials", "brute_force_seq",
+    "attention_row", "attention_row_grad", "partial_attention", "merge_partials", "brute_force_seq",
 ]
 
 
@@ -148,6 +148,21 @@ def attention_row(q_i, k, v, i):
     e = np.exp(s - m)
     z = e.sum()
     return (e / z) @ v[: i + 1], m + math.log(z)
+
+
+def attention_row_grad(q_i, k, v, do_i, i):
+    """Gradient terms of a single query row i of one (sequence, head): returns (dq_i[D], p[i+1],
+    ds[i+1]); row i adds p_j * dO_i to dv_j and ds_j * q_i / sqrt(D) to dk_j for every j <= i."""
+    D = q_i.shape[-1]
+    s = (k[: i + 1] @ q_i) / math.sqrt(D)
+    m = s.max()
+    e = np.exp(s - m)
+    p = e / e.sum()
+    o_i = p @ v[: i + 1]
+    dp = v[: i + 1] @ do_i
+    delta = float(do_i @ o_i)
+    ds = p * (dp - delta)
+    return (ds @ k[: i + 1]) / math.sqrt(D), p, ds
 
 
 def partial_attention(q, k, v, q_rows, kv_ranges):

@@ -65,6 +65,26 @@ int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int D, int 
   return FCP_OK;
 }
 
+// Records an event pair around a kernel launch when the plan is in profiling mode.
+struct ProfScope {
+  const fcp_plan* plan;
+  int kind;
+  cudaStream_t st;
+  int slot = -1;
+  ProfScope(const fcp_plan* p, int k, cudaStream_t s) : plan(p), kind(k), st(s) {
+    if (plan->profiling && plan->prof_ev[kind][0][0]) {
+      slot = (int)(plan->prof_n[kind] % 64);
+      cudaEventRecord((cudaEvent_t)plan->prof_ev[kind][slot][0], st);
+    }
+  }
+  ~ProfScope() {
+    if (slot >= 0) {
+      cudaEventRecord((cudaEvent_t)plan->prof_ev[kind][slot][1], st);
+      ++plan->prof_n[kind];
+    }
+  }
+};
+
 int check_plan(const fcp_plan* plan) {
   if (!plan) {
     fcp_set_error("plan is NULL");
@@ -87,7 +107,7 @@ template <int D>
 __global__ void __launch_bounds__(256) fcp_merge_kernel(const int32_t* __restrict__ units, const int32_t* __restrict__ slot_offset,
                                                         const int32_t* __restrict__ slot_rows, const float* __restrict__ o_partial,
                                                         const float* __restrict__ lse_partial, int head_begin, int head_count,
-                                                        int hq, __nv_bfloat16* __restrict__ o, float* __restrict__ lse) {
+                                                        int hq, __nv_bfloat16* __restrict__ o, float* __restrict__ o_f32, float* __restrict__ lse) {
   constexpr int TPR = D / 8;                 // threads per (token, head) row
   constexpr int RPP = 256 / TPR;             // rows per pass
   const int32_t* U = units + (size_t)blockIdx.x * FCP_MERGE_UNIT_W;
@@ -118,6 +138,11 @@ __global__ void __launch_bounds__(256) fcp_merge_kernel(const int32_t* __restric
     pk.x = pack_bf16(acc[0], acc[1]); pk.y = pack_bf16(acc[2], acc[3]);
     pk.z = pack_bf16(acc[4], acc[5]); pk.w = pack_bf16(acc[6], acc[7]);
     *reinterpret_cast<uint4*>(o + orow * D + sub * 8) = pk;
+    if (o_f32) {
+      float4* dst = reinterpret_cast<float4*>(o_f32 + orow * D + sub * 8);
+      dst[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+      dst[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    }
     if (sub == 0) lse[orow] = L;
   }
 }
@@ -222,8 +247,43 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   return FCP_OK;
 }
 
+extern "C" int fcp_plan_set_profiling(fcp_plan* plan, int32_t enable) {
+  if (!plan) return FCP_ERR_INVALID_ARG;
+  for (int k = 0; k < FCP_KERNEL_KINDS; ++k) {
+    plan->prof_n[k] = 0;
+    for (int i = 0; i < 64; ++i)
+      for (int e = 0; e < 2; ++e) {
+        if (enable && !plan->prof_ev[k][i][e]) {
+          cudaEvent_t ev;
+          FCP_CUDA_CHECK(cudaEventCreate(&ev));
+          plan->prof_ev[k][i][e] = ev;
+        } else if (!enable && plan->prof_ev[k][i][e]) {
+          cudaEventDestroy((cudaEvent_t)plan->prof_ev[k][i][e]);
+          plan->prof_ev[k][i][e] = nullptr;
+        }
+      }
+  }
+  plan->profiling = enable != 0;
+  return FCP_OK;
+}
+
+extern "C" int fcp_plan_kernel_ms(const fcp_plan* plan, int32_t kind, int32_t* launches, float* mean_ms) {
+  if (!plan || kind < 0 || kind >= FCP_KERNEL_KINDS || !launches || !mean_ms) return FCP_ERR_INVALID_ARG;
+  const int n = (int)std::min<int64_t>(plan->prof_n[kind], 64);
+  double sum = 0.0;
+  for (int i = 0; i < n; ++i) {
+    float ms = 0.f;
+    FCP_CUDA_CHECK(cudaEventElapsedTime(&ms, (cudaEvent_t)plan->prof_ev[kind][i][0], (cudaEvent_t)plan->prof_ev[kind][i][1]));
+    sum += ms;
+  }
+  *launches = (int32_t)plan->prof_n[kind];
+  *mean_ms = n ? (float)(sum / n) : 0.f;
+  return FCP_OK;
+}
+
 extern "C" int fcp_plan_destroy(fcp_plan* plan) {
   if (!plan) return FCP_OK;
+  fcp_plan_set_profiling(plan, 0);
   if (plan->d_blob) cudaFree(plan->d_blob);
   delete plan;
   return FCP_OK;
@@ -295,6 +355,7 @@ extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, 
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
   if (grid == 0) return FCP_OK;
   cudaStream_t st = (cudaStream_t)stream;
+  ProfScope prof(plan, 0, st);
   if (P.head_dim == 128)
     fcp_fwd_kernel<128><<<grid, FWD_THREADS, FwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, a);
   else
@@ -304,7 +365,8 @@ extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, 
 }
 
 extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
-                             int32_t head_begin, int32_t head_count, void* o, float* lse, void* stream) {
+                             int32_t head_begin, int32_t head_count, void* o, float* o_f32, float* lse,
+                             void* stream) {
   int rc = check_plan(plan);
   if (rc != FCP_OK) return rc;
   if (!o_partial || !lse_partial || !o || !lse) {
@@ -316,12 +378,13 @@ extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const
   const int n_units = (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W);
   if (n_units == 0) return FCP_OK;
   cudaStream_t st = (cudaStream_t)stream;
+  ProfScope prof(plan, 1, st);
   if (P.head_dim == 128)
     fcp_merge_kernel<128><<<n_units, 256, 0, st>>>(plan->d_merge_units, plan->d_slot_offset, plan->d_slot_rows, o_partial,
-                                                   lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, lse);
+                                                   lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, o_f32, lse);
   else
     fcp_merge_kernel<64><<<n_units, 256, 0, st>>>(plan->d_merge_units, plan->d_slot_offset, plan->d_slot_rows, o_partial,
-                                                  lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, lse);
+                                                  lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, o_f32, lse);
   FCP_CUDA_CHECK(cudaGetLastError());
   return FCP_OK;
 }
@@ -348,8 +411,9 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   float* dq_acc = (float*)scratch;
   float* delta_t = dq_acc + T * P.hq * D;
   float* lse2_t = delta_t + tpad * P.hq;
-  FCP_CUDA_CHECK(cudaMemsetAsync(scratch, 0, (size_t)need, st));
   {
+    ProfScope prof(plan, 2, st);
+    FCP_CUDA_CHECK(cudaMemsetAsync(scratch, 0, (size_t)need, st));
     const int64_t rows = T * P.hq;
     const int tpr = (int)D / 8;
     const int64_t blocks = (rows * tpr + 255) / 256;
@@ -385,6 +449,7 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   const int64_t n_work = (int64_t)a.n_units * P.hkv;
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
   if (grid > 0) {
+    ProfScope prof(plan, 3, st);
     if (D == 128)
       fcp_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
     else
@@ -394,6 +459,7 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   {
     const int64_t n8 = T * P.hq * D / 8;
     const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)plan->sm_count * 16);
+    ProfScope prof(plan, 4, st);
     fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8);
     FCP_CUDA_CHECK(cudaGetLastError());
   }
@@ -480,7 +546,7 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
     const int hc = std::min(L.heads_per_pass, P.hq - h0);
     if ((rc = fcp_attn_fwd(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part), st)) != FCP_OK)
       return rc;
-    if ((rc = fcp_lse_merge(plan, (float*)(w + L.o_part), (float*)(w + L.lse_part), h0, hc, w + L.o, (float*)(w + L.lse), st)) != FCP_OK)
+    if ((rc = fcp_lse_merge(plan, (float*)(w + L.o_part), (float*)(w + L.lse_part), h0, hc, w + L.o, nullptr, (float*)(w + L.lse), st)) != FCP_OK)
       return rc;
   }
   int64_t scratch = 0;

@@ -43,6 +43,11 @@ struct fcp_plan {
   int32_t* d_slot_rows = nullptr;
   int32_t* d_status = nullptr; // [4]: status word, diagnostic
   int sm_count = 0;
+
+  // optional kernel timing: ring of event pairs per kernel kind (void* = cudaEvent_t)
+  bool profiling = false;
+  void* prof_ev[FCP_KERNEL_KINDS][64][2] = {};
+  mutable int64_t prof_n[FCP_KERNEL_KINDS] = {};
 };
 
 void fcp_set_error(const char* fmt, ...);

@@ -25,7 +25,8 @@ INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merg
 
 EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
            "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_lse_merge", "fcp_attn_bwd",
-           "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_status_string",
+           "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
+           "fcp_plan_kernel_ms", "fcp_status_string",
            "fcp_last_error_message"]
 
 
@@ -66,10 +67,12 @@ def lib() -> C.CDLL:
     L.fcp_plan_upload.argtypes = [vp, vp]
     L.fcp_plan_destroy.argtypes = [vp]
     L.fcp_attn_fwd.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp]
-    L.fcp_lse_merge.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp]
-    L.fcp_attn_bwd.argtypes = [vp] + [vp] * 11 + [C.c_int64, vp]
+    L.fcp_lse_merge.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
+    L.fcp_plan_set_profiling.argtypes = [vp, C.c_int32]
+    L.fcp_plan_kernel_ms.argtypes = [vp, C.c_int32, i32p, f32p]
+    L.fcp_attn_bwd.argtypes = [vp] * 11 + [C.c_int64, vp]
     L.fcp_host_workspace_bytes.argtypes = [vp, i64p]
-    L.fcp_attn_fwd_bwd_host.argtypes = [vp] + [vp] * 10 + [C.c_int64, vp]
+    L.fcp_attn_fwd_bwd_host.argtypes = [vp] * 11 + [C.c_int64, vp]
     L.fcp_last_device_status.argtypes = [vp, i32p]
     L.fcp_status_string.argtypes = [C.c_int]
     L.fcp_status_string.restype = C.c_char_p
@@ -169,6 +172,15 @@ class Plan:
         _check(lib().fcp_plan_upload(self.handle, C.c_void_p(stream)))
         return self
 
+    def set_profiling(self, enable: bool):
+        _check(lib().fcp_plan_set_profiling(self.handle, 1 if enable else 0))
+
+    def kernel_ms(self, kind: int):
+        n = C.c_int32(0)
+        ms = C.c_float(0.0)
+        _check(lib().fcp_plan_kernel_ms(self.handle, int(kind), C.byref(n), C.byref(ms)))
+        return n.value, ms.value
+
     def device_status(self):
         st = np.zeros(4, dtype=np.int32)
         _check(lib().fcp_last_device_status(self.handle, st.ctypes.data_as(C.POINTER(C.c_int32))))
@@ -185,10 +197,10 @@ def fcp_attn_fwd(plan: Plan, q, k, v, o_partial, lse_partial, head_begin=0, head
                               _ptr(lse_partial), C.c_void_p(stream)))
 
 
-def fcp_lse_merge(plan: Plan, o_partial, lse_partial, o, lse, head_begin=0, head_count=None, stream=0):
+def fcp_lse_merge(plan: Plan, o_partial, lse_partial, o, lse, head_begin=0, head_count=None, stream=0, o_f32=None):
     hc = plan.hq - head_begin if head_count is None else head_count
     _check(lib().fcp_lse_merge(plan.handle, _ptr(o_partial), _ptr(lse_partial), int(head_begin), int(hc), _ptr(o),
-                               _ptr(lse), C.c_void_p(stream)))
+                               _ptr(o_f32), _ptr(lse), C.c_void_p(stream)))
 
 
 def fcp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, scratch, scratch_bytes, stream=0):

@@ -1,0 +1,285 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle on the same seeded inputs.
+
+Tolerances (stated for bf16 inputs with fp32 accumulation):
+  O    max abs <= 1e-2, mean abs <= 1e-3     (checked on the fp32 output; the bf16 copy of O is
+                                             allowed its own rounding, half an ulp = 2^-8 * |o|, on top)
+  LSE  max abs <= 1e-3
+  dQ, dK, dV   relative Frobenius error <= 2e-2
+  plan tables  bit-exact (tests/test_host_plan.py, host only)
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import attention_ref as A
+from oracle import plan_ref as P
+from paper_2602_21788_b200 import build, synth
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+O_MAX, O_MEAN, LSE_MAX, GRAD_REL = 1e-2, 1e-3, 1e-3, 2e-2
+f64 = synth.bf16_bits_to_f64
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _gpu():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    build.build()
+    torch.cuda.set_device(0)
+
+
+def _wl(lens, degs, hq, hkv, D, seed=0):
+    return synth.Workload(name="case", seed=seed, seqlens=np.asarray(lens, np.int32),
+                          cp_degrees=np.asarray(degs, np.int32), hq=hq, hkv=hkv, head_dim=D)
+
+
+def _grad_ok(got, ref):
+    """Relative Frobenius error <= 2e-2; the absolute floor only matters where the exact gradient is
+    zero (a single-token sequence has dq = dk = 0) and the ratio is undefined."""
+    err = np.linalg.norm(np.asarray(got, dtype=np.float64) - ref)
+    return err <= GRAD_REL * np.linalg.norm(ref) + 1e-4 * math.sqrt(ref.size), err / max(np.linalg.norm(ref), 1e-300)
+
+
+def _check_full(w, heads_per_pass=None, bwd=True, check_partials=False):
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    q, k, v, do = w.tensors()
+    res = run_fwd_bwd(w, q, k, v, do if bwd else None, heads_per_pass=heads_per_pass, keep_partials=check_partials)
+    qf, kf, vf, dof = f64(q), f64(k), f64(v), f64(do)
+    o_ref, lse_ref = A.attention_fwd_packed(qf, kf, vf, w.cu_seqlens)
+    e = np.abs(res["o_f32"] - o_ref)
+    assert e.max() <= O_MAX and e.mean() <= O_MEAN, (e.max(), e.mean())
+    eb = np.abs(res["o"] - o_ref)
+    assert np.all(eb <= O_MAX + np.abs(o_ref) * 2.0 ** -8) and eb.mean() <= O_MEAN, (eb.max(), eb.mean())
+    assert np.abs(res["lse"] - lse_ref).max() <= LSE_MAX
+    if check_partials:
+        _check_partials(w, res, qf, kf, vf)
+    if bwd:
+        dq_ref, dk_ref, dv_ref = A.attention_bwd_packed(qf, kf, vf, dof, w.cu_seqlens)
+        for name, ref in (("dq", dq_ref), ("dk", dk_ref), ("dv", dv_ref)):
+            ok, rel = _grad_ok(res[name], ref)
+            assert ok, (name, rel)
+            assert np.isfinite(res[name]).all()
+    return res
+
+
+def _check_partials(w, res, qf, kf, vf):
+    """Every item's normalised partial and its LSE against the oracle's partial over the same KV ranges."""
+    lens, degs = w.seqlens.tolist(), w.cp_degrees.tolist()
+    pl = P.plan_blocks(lens, degs)
+    cb, co = pl["chunk_bounds"], pl["chunk_offset"]
+    g = w.hq // w.hkv
+    for (b, r, s, qc, slot, row0, n, first) in pl["items"]:
+        t0 = cb[co[b]]
+        qr = (cb[co[b] + qc] - t0, cb[co[b] + qc + 1] - t0)
+        ranges = [(cb[co[b] + kc] - t0, cb[co[b] + kc + 1] - t0) for (_, _, _, _, kc, _) in pl["pairs"][first:first + n]]
+        sl = slice(t0, t0 + lens[b])
+        for h in range(w.hq):
+            op, lp = A.partial_attention(qf[sl, h], kf[sl, h // g], vf[sl, h // g], qr, ranges)
+            rows = slice(row0, row0 + qr[1] - qr[0])
+            assert np.abs(res["o_partial"][rows, h] - op).max() <= O_MAX
+            assert np.abs(res["lse_partial"][rows, h] - lp).max() <= LSE_MAX
+
+
+EDGE_CASES = [
+    # lens, degs, hq, hkv, D
+    ([1], [1], 1, 1, 128),                    # single token
+    ([1, 2, 3], [3, 2, 4], 2, 1, 64),         # L < 2d: empty chunks are dropped
+    ([128], [1], 1, 1, 128),                  # exactly one tile
+    ([129], [1], 2, 2, 64),                   # one row into the second tile
+    ([256, 257, 255], [1, 1, 1], 2, 1, 128),  # around the two-tile unit
+    ([100], [8], 4, 4, 64),                   # chunks shorter than a tile (6-7 tokens)
+    ([1000], [7], 8, 1, 128),                 # non-power-of-two degree, GQA 8:1, L % 14 != 0
+    ([1031], [5], 4, 2, 128),                 # prime length
+    ([777, 64, 1500], [3, 1, 6], 4, 4, 64),   # hq == hkv
+    ([2048], [8], 2, 1, 128),                 # d = 8, chunk = one tile exactly
+    ([3000], [1], 2, 1, 128),                 # d = 1: plain varlen causal attention
+    ([513], [64], 1, 1, 64),                  # largest supported degree
+]
+
+
+@pytest.mark.parametrize("lens,degs,hq,hkv,D", EDGE_CASES)
+def test_edge_shapes(lens, degs, hq, hkv, D):
+    _check_full(_wl(lens, degs, hq, hkv, D, seed=3), check_partials=True)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_tiny_workload(seed):
+    _check_full(synth.make_workload("tiny", seed), check_partials=True)
+
+
+@pytest.mark.parametrize("name", ["llama8b_64k", "longtail_256k", "bimodal_128k", "extreme_512k"])
+def test_reduced_workloads(name):
+    """Same generators and degrees, lengths / 16, at most 8 query heads: the oracle runs in full."""
+    w = synth.reduced(synth.make_workload(name, 0))
+    _check_full(w)
+
+
+def test_head_passes_give_the_same_result():
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = _wl([700, 300], [3, 2], 8, 2, 128, seed=5)
+    q, k, v, do = w.tensors()
+    a = run_fwd_bwd(w, q, k, v, do)
+    b = run_fwd_bwd(w, q, k, v, do, heads_per_pass=3)
+    assert np.array_equal(a["o"], b["o"]) and np.array_equal(a["lse"], b["lse"])
+
+
+def test_forward_and_merge_are_bitwise_reproducible_and_backward_within_tolerance():
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = synth.make_workload("tiny", 1)
+    q, k, v, do = w.tensors()
+    a = run_fwd_bwd(w, q, k, v, do)
+    b = run_fwd_bwd(w, q, k, v, do)
+    assert np.array_equal(a["o"], b["o"]) and np.array_equal(a["lse"], b["lse"]) and np.array_equal(a["o_f32"], b["o_f32"])
+    assert np.array_equal(a["dk"], b["dk"]) and np.array_equal(a["dv"], b["dv"])   # no atomics on dK/dV
+    assert np.linalg.norm(a["dq"] - b["dq"]) <= 1e-2 * np.linalg.norm(a["dq"])       # fp32 atomics: order varies
+
+
+def test_chunked_plan_agrees_with_degree_one_plan():
+    """Self-consistency without the oracle: the configured degrees vs all d = 1."""
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = synth.reduced(synth.make_workload("bimodal_128k", 1), len_div=8)
+    q, k, v, do = w.tensors()
+    a = run_fwd_bwd(w, q, k, v, do)
+    w1 = _wl(w.seqlens, np.ones_like(w.cp_degrees), w.hq, w.hkv, w.head_dim, seed=w.seed)
+    w1.name = w.name
+    b = run_fwd_bwd(w1, q, k, v, do)
+    assert np.abs(a["o_f32"] - b["o_f32"]).max() <= O_MAX and np.abs(a["lse"] - b["lse"]).max() <= LSE_MAX
+    for n in ("dq", "dk", "dv"):
+        assert np.linalg.norm(a[n] - b[n]) <= GRAD_REL * np.linalg.norm(b[n])
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    from paper_2602_21788_b200 import fcp
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = _wl([900, 130], [3, 1], 4, 2, 128, seed=7)
+    q, k, v, do = w.tensors()
+    ref = run_fwd_bwd(w, q, k, v, do)
+    plan = ref["state"].plan
+    T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
+    pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
+    hq_, hk_, hv_, hdo_ = pin(q), pin(k), pin(v), pin(do)
+    ho = torch.empty((T, hq, D), dtype=torch.int16).pin_memory()
+    hdq = torch.empty((T, hq, D), dtype=torch.int16).pin_memory()
+    hdk = torch.empty((T, hkv, D), dtype=torch.int16).pin_memory()
+    hdv = torch.empty((T, hkv, D), dtype=torch.int16).pin_memory()
+    hlse = torch.empty((T, hq), dtype=torch.float32).pin_memory()
+    nbytes = plan.host_workspace_bytes()
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    fcp.fcp_attn_fwd_bwd_host(plan, hq_, hk_, hv_, hdo_, ho, hlse, hdq, hdk, hdv, ws, nbytes,
+                              torch.cuda.current_stream().cuda_stream)
+    back = lambda t: f64(t.numpy().view(np.uint16))
+    assert np.array_equal(back(ho), ref["o"]) and np.array_equal(hlse.numpy(), ref["lse"])
+    assert np.array_equal(back(hdk), ref["dk"]) and np.array_equal(back(hdv), ref["dv"])
+    assert np.linalg.norm(back(hdq) - ref["dq"]) <= 1e-2 * np.linalg.norm(ref["dq"])
+    with pytest.raises(fcp.FcpError) as e:
+        fcp.fcp_attn_fwd_bwd_host(plan, hq_, hk_, hv_, hdo_, ho, hlse, hdq, hdk, hdv, ws, 1024, 0)
+    assert e.value.status == fcp.FCP_ERR_WORKSPACE
+
+
+def test_workspace_too_small_is_reported():
+    from paper_2602_21788_b200 import fcp
+    from paper_2602_21788_b200.runner import DeviceState
+    w = _wl([300], [1], 2, 1, 128)
+    q, k, v, do = w.tensors()
+    ds = DeviceState(w, q, k, v, do)
+    ds.forward()
+    with pytest.raises(fcp.FcpError) as e:
+        fcp.fcp_attn_bwd(ds.plan, ds.q, ds.k, ds.v, ds.o, ds.do, ds.lse, ds.dq, ds.dk, ds.dv, ds.scratch, 16, 0)
+    assert e.value.status == fcp.FCP_ERR_WORKSPACE
+    with pytest.raises(fcp.FcpError) as e:
+        fcp.fcp_attn_fwd(ds.plan, ds.q, ds.k, ds.v, ds.o_part, ds.lse_part, 1, 2, 0)   # heads [1,3) of 2
+    assert e.value.status == fcp.FCP_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+
+
+# ----------------------------------------------------------------------------------------------
+# Full-size workloads: the oracle evaluates sampled outputs one by one.
+# ----------------------------------------------------------------------------------------------
+def _sampled_check(w, n_rows=96, n_tail=24, seed=0):
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    q, k, v, do = w.tensors()
+    res = run_fwd_bwd(w, q, k, v, do)
+    rng = np.random.default_rng(seed)
+    cu = w.cu_seqlens
+    g = w.hq // w.hkv
+    D = w.head_dim
+    longest = int(np.argmax(w.seqlens))
+    # forward rows and dQ rows: random (sequence, token, head), biased to long sequences and chunk edges
+    o_err, l_err, dq_num, dq_den = [], [], 0.0, 0.0
+    for n in range(n_rows):
+        b = longest if n % 3 == 0 else int(rng.integers(len(w.seqlens)))
+        L = int(w.seqlens[b])
+        i = int(rng.integers(L)) if n % 4 else L - 1 - int(rng.integers(min(L, 300)))
+        h = int(rng.integers(w.hq))
+        t0 = int(cu[b])
+        ks, vs = f64(k[t0:t0 + i + 1, h // g]), f64(v[t0:t0 + i + 1, h // g])
+        qi, doi = f64(q[t0 + i, h]), f64(do[t0 + i, h])
+        o_ref, lse_ref = A.attention_row(qi, ks, vs, i)
+        dq_ref, _, _ = A.attention_row_grad(qi, ks, vs, doi, i)
+        o_err.append(np.abs(res["o_f32"][t0 + i, h] - o_ref))
+        l_err.append(abs(res["lse"][t0 + i, h] - lse_ref))
+        dq_num += np.sum((res["dq"][t0 + i, h] - dq_ref) ** 2)
+        dq_den += np.sum(dq_ref ** 2)
+    o_err = np.concatenate(o_err)
+    assert o_err.max() <= O_MAX and o_err.mean() <= O_MEAN, (o_err.max(), o_err.mean())
+    assert max(l_err) <= LSE_MAX
+    assert math.sqrt(dq_num / dq_den) <= GRAD_REL
+    # dK/dV columns: the last n_tail tokens of the longest sequence (every later row of every head of
+    # the group contributes), one KV head
+    b, L, t0 = longest, int(w.seqlens[longest]), int(cu[longest])
+    hk = int(rng.integers(w.hkv))
+    ks, vs = f64(k[t0:t0 + L, hk]), f64(v[t0:t0 + L, hk])
+    j0 = L - n_tail
+    dk_ref = np.zeros((n_tail, D)); dv_ref = np.zeros((n_tail, D))
+    for h in range(hk * g, hk * g + g):
+        for i in range(j0, L):
+            qi, doi = f64(q[t0 + i, h]), f64(do[t0 + i, h])
+            _, p, ds = A.attention_row_grad(qi, ks, vs, doi, i)
+            dv_ref[: i - j0 + 1] += p[j0:, None] * doi[None, :]
+            dk_ref[: i - j0 + 1] += ds[j0:, None] * qi[None, :] / math.sqrt(D)
+    for name, ref in (("dk", dk_ref), ("dv", dv_ref)):
+        got = res[name][t0 + j0:t0 + L, hk]
+        assert np.linalg.norm(got - ref) <= GRAD_REL * np.linalg.norm(ref), name
+    # one whole short sequence in full
+    short = [b for b in range(len(w.seqlens)) if w.seqlens[b] <= 1536]
+    if short:
+        b = short[0]
+        t0, t1 = int(cu[b]), int(cu[b + 1])
+        sub_cu = np.array([0, t1 - t0])
+        qf, kf, vf, dof = f64(q[t0:t1]), f64(k[t0:t1]), f64(v[t0:t1]), f64(do[t0:t1])
+        o_ref, lse_ref = A.attention_fwd_packed(qf, kf, vf, sub_cu)
+        dq_ref, dk_ref, dv_ref = A.attention_bwd_packed(qf, kf, vf, dof, sub_cu)
+        e = np.abs(res["o_f32"][t0:t1] - o_ref)
+        assert e.max() <= O_MAX and e.mean() <= O_MEAN
+        assert np.abs(res["lse"][t0:t1] - lse_ref).max() <= LSE_MAX
+        for name, ref in (("dq", dq_ref), ("dk", dk_ref), ("dv", dv_ref)):
+            assert np.linalg.norm(res[name][t0:t1] - ref) <= GRAD_REL * np.linalg.norm(ref), name
+    # properties that hold at any size
+    assert np.isfinite(res["o"]).all() and np.isfinite(res["lse"]).all()
+    for n in ("dq", "dk", "dv"):
+        assert np.isfinite(res[n]).all()
+    first = cu[:-1]
+    assert np.array_equal(res["o"][first], np.repeat(f64(v[first]), g, axis=1))   # first token attends to itself only
+
+
+def test_full_size_llama8b_64k_sampled():
+    """The configuration the benchmark times (all heads in one pass)."""
+    _sampled_check(synth.make_workload("llama8b_64k", 0))
+
+
+@pytest.mark.slow
+def test_full_size_bimodal_128k_sampled():
+    _sampled_check(synth.make_workload("bimodal_128k", 0), n_rows=48, n_tail=8)
+
+
+@pytest.mark.slow
+def test_full_length_extreme_with_eight_heads_sampled():
+    """Full 512K-token lengths (one 384K sequence, degree 7), 8 query heads on 1 KV head: exercises the
+    64-bit offsets and the long-tail schedule while the inputs still fit the host quickly."""
+    w = synth.make_workload("extreme_512k", 0)
+    w.hq, w.hkv = 8, 1
+    _sampled_check(w, n_rows=32, n_tail=4)

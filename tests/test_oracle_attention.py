@@ -136,6 +136,19 @@ def test_row_slabs_and_row_form_agree_with_full_form():
         assert np.allclose(oi, o[i], atol=1e-13) and math.isclose(li, lse[i], rel_tol=1e-13)
 
 
+def test_row_gradient_form_sums_to_full_gradients():
+    L, D = 40, 8
+    q, k, v, do = _rand(L, D, 14)
+    dq, dk, dv = A.attention_bwd_seq(q, k, v, do)
+    dk2 = np.zeros_like(dk); dv2 = np.zeros_like(dv)
+    for i in range(L):
+        dqi, p, ds = A.attention_row_grad(q[i], k, v, do[i], i)
+        assert np.allclose(dqi, dq[i], atol=1e-13)
+        dv2[: i + 1] += p[:, None] * do[i][None, :]
+        dk2[: i + 1] += ds[:, None] * q[i][None, :] / math.sqrt(D)
+    assert np.allclose(dk2, dk, atol=1e-12) and np.allclose(dv2, dv, atol=1e-12)
+
+
 def test_packed_gqa_matches_per_sequence_and_sums_kv_heads():
     rng = np.random.default_rng(12)
     lens = [5, 1, 19]
