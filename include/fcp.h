@@ -105,6 +105,7 @@ int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B
 #define FCP_TABLE_BWD_UNITS     8  /* [n_bwd_units][8]          derived                               */
 #define FCP_TABLE_BWD_QRANGES   9  /* [n_bwd_qranges][4]        derived                               */
 #define FCP_TABLE_MERGE_UNITS  10  /* [n_merge_units][4]        derived                               */
+#define FCP_TABLE_BWD_WORK     11  /* [n_bwd_units*hkv][2]      derived: (unit, kv head) in execution order */
 
 /* fcp_plan_get: *host_ptr = first element of the table, *count = number of int32 elements. */
 int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count);

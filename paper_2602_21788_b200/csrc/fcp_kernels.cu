@@ -148,12 +148,12 @@ __global__ void __launch_bounds__(256) fcp_merge_kernel(const int32_t* __restric
 }
 
 // ---------------------------------------------------------------------------------------------
-// Backward preprocess (HBM bound): delta[h][t] = sum_c dO[t,h,c] * O[t,h,c], and the forward LSE
+// Backward preprocess (HBM bound): delta[h][t] = scale * sum_c dO[t,h,c] * O[t,h,c], and the forward LSE
 // transposed to [h][t] in log2 units, the layout the backward kernel's per-tile loads want.
 // ---------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) fcp_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
-                                                        const float* __restrict__ lse, int64_t T, int hq, int64_t t_stride,
+                                                        const float* __restrict__ lse, int64_t T, int hq, int64_t t_stride, float scale,
                                                         float* __restrict__ delta_t, float* __restrict__ lse2_t) {
   constexpr int TPR = D / 8;
   const int64_t row = ((int64_t)blockIdx.x * 256 + threadIdx.x) / TPR;   // (token, head) row
@@ -175,7 +175,7 @@ __global__ void __launch_bounds__(256) fcp_delta_kernel(const __nv_bfloat16* __r
   if (row < T * hq && sub == 0) {
     const int64_t t = row / hq;
     const int h = (int)(row % hq);
-    delta_t[h * t_stride + t] = acc;
+    delta_t[h * t_stride + t] = acc * scale;
     lse2_t[h * t_stride + t] = lse[row] * 1.4426950408889634f;
   }
 }
@@ -209,20 +209,20 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   }
   plan->device = dev;
   plan->sm_count = prop.multiProcessorCount;
-  const std::vector<int32_t>* tabs[6] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges,
-                                         &plan->merge_units, &plan->slot_offset, &plan->slot_rows};
-  size_t off[7];
+  const std::vector<int32_t>* tabs[7] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges,
+                                         &plan->merge_units, &plan->slot_offset, &plan->slot_rows, &plan->bwd_work};
+  size_t off[8];
   size_t total = 256;  // status words first
-  for (int i = 0; i < 6; ++i) {
+  for (int i = 0; i < 7; ++i) {
     off[i] = total;
     total += (tabs[i]->size() * 4 + 255) / 256 * 256;
   }
-  off[6] = total;
+  off[7] = total;
   void* blob = nullptr;
   FCP_CUDA_CHECK(cudaMalloc(&blob, total));
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(blob, 0, 256, st);
-  for (int i = 0; i < 6 && e == cudaSuccess; ++i)
+  for (int i = 0; i < 7 && e == cudaSuccess; ++i)
     if (!tabs[i]->empty())
       e = cudaMemcpyAsync((char*)blob + off[i], tabs[i]->data(), tabs[i]->size() * 4, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -239,6 +239,7 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   plan->d_merge_units = (int32_t*)((char*)blob + off[3]);
   plan->d_slot_offset = (int32_t*)((char*)blob + off[4]);
   plan->d_slot_rows = (int32_t*)((char*)blob + off[5]);
+  plan->d_bwd_work = (int32_t*)((char*)blob + off[6]);
   // opt in to the large dynamic shared memory of the tensor-core kernels once
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::DYN_BYTES));
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::DYN_BYTES));
@@ -414,15 +415,16 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   {
     ProfScope prof(plan, 2, st);
     FCP_CUDA_CHECK(cudaMemsetAsync(scratch, 0, (size_t)need, st));
+    FCP_CUDA_CHECK(cudaMemsetAsync(plan->d_status + 16, 0, sizeof(int32_t), st));   // work counter of the backward grid
     const int64_t rows = T * P.hq;
     const int tpr = (int)D / 8;
     const int64_t blocks = (rows * tpr + 255) / 256;
     if (D == 128)
       fcp_delta_kernel<128><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                              tpad, delta_t, lse2_t);
+                                                              tpad, P.scale, delta_t, lse2_t);
     else
       fcp_delta_kernel<64><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                             tpad, delta_t, lse2_t);
+                                                             tpad, P.scale, delta_t, lse2_t);
     FCP_CUDA_CHECK(cudaGetLastError());
   }
   CUtensorMap tq, tk, tv, tdo;
@@ -433,7 +435,9 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   BwdArgs a;
   a.units = plan->d_bwd_units;
   a.qranges = plan->d_bwd_qranges;
-  a.n_units = (int32_t)(plan->bwd_units.size() / FCP_BWD_UNIT_W);
+  a.work = plan->d_bwd_work;
+  a.n_work = (int32_t)(plan->bwd_work.size() / 2);
+  a.counter = plan->d_status + 16;
   a.hq = P.hq;
   a.hkv = P.hkv;
   a.T = T;
@@ -446,8 +450,7 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   a.dk = (__nv_bfloat16*)dk;
   a.dv = (__nv_bfloat16*)dv;
   a.status = plan->d_status;
-  const int64_t n_work = (int64_t)a.n_units * P.hkv;
-  const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
+  const int grid = (int)std::min<int64_t>(a.n_work, plan->sm_count);
   if (grid > 0) {
     ProfScope prof(plan, 3, st);
     if (D == 128)

@@ -380,8 +380,25 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
       }
     }
   }
-  std::stable_sort(bus.begin(), bus.end(), [](const BU& a, const BU& b) { return a.f[BU_COST] > b.f[BU_COST]; });
   for (const BU& u : bus) p->bwd_units.insert(p->bwd_units.end(), u.f, u.f + FCP_BWD_UNIT_W);
+  // Execution order of the backward work items (unit, KV head).  dQ is accumulated with fp32
+  // reductions in global memory, which only run at L2 speed while the rows they touch stay
+  // resident: so all CTAs work on one (sequence, KV head) panel at a time, key tiles in ascending
+  // position (descending cost), and sweep the query tiles roughly in step.  Sequences go longest
+  // first, which leaves the small units for the tail of the schedule.
+  {
+    std::vector<int> seq_order(B);
+    std::iota(seq_order.begin(), seq_order.end(), 0);
+    std::stable_sort(seq_order.begin(), seq_order.end(), [&](int a, int b) { return seqlens[a] > seqlens[b]; });
+    std::vector<std::vector<int32_t>> units_of(B);
+    for (size_t i = 0; i < bus.size(); ++i) units_of[bus[i].f[BU_SEQ]].push_back((int32_t)i);   // ascending key position
+    for (int b : seq_order)
+      for (int hk = 0; hk < params->hkv; ++hk)
+        for (int32_t u : units_of[b]) {
+          p->bwd_work.push_back(u);
+          p->bwd_work.push_back(hk);
+        }
+  }
 
   // Merge: runs of up to FCP_MERGE_TOKENS tokens inside one chunk.
   for (int b = 0; b < B; ++b) {
@@ -411,6 +428,7 @@ extern "C" int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t**
     case FCP_TABLE_BWD_UNITS: v = &plan->bwd_units; break;
     case FCP_TABLE_BWD_QRANGES: v = &plan->bwd_qranges; break;
     case FCP_TABLE_MERGE_UNITS: v = &plan->merge_units; break;
+    case FCP_TABLE_BWD_WORK: v = &plan->bwd_work; break;
     default: fcp_set_error("fcp_plan_get: unknown table %d", which); return FCP_ERR_INVALID_ARG;
   }
   *host_ptr = v->data();

@@ -30,7 +30,7 @@ struct fcp_plan {
   int64_t T = 0;   // total tokens
   int64_t R = 0;   // rows of the partial buffers
   std::vector<int32_t> cu_seqlens, chunk_offset, chunk_bounds, pairs, items, slot_offset, slot_rows;
-  std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units;
+  std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units, bwd_work;
 
   // device copy (fcp_plan_upload)
   int device = -1;
@@ -39,6 +39,7 @@ struct fcp_plan {
   int32_t* d_bwd_units = nullptr;
   int32_t* d_bwd_qranges = nullptr;
   int32_t* d_merge_units = nullptr;
+  int32_t* d_bwd_work = nullptr;
   int32_t* d_slot_offset = nullptr;
   int32_t* d_slot_rows = nullptr;
   int32_t* d_status = nullptr; // [4]: status word, diagnostic

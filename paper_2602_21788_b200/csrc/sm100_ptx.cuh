@@ -61,14 +61,15 @@ struct WaitCtx {
 
 // Bounded wait.  Returns false if the CTA is aborting (this waiter timed out, or another did).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, int where) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
   uint32_t spins = 0;
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((++spins & 255u) == 0) {
+  unsigned long long t0 = 0;
+#pragma unroll 1
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 1023u) == 0) {
       if (*ctx.abort_flag) return false;
-      if (globaltimer_ns() - t0 > FCP_WAIT_NS) {
+      const unsigned long long now = globaltimer_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > FCP_WAIT_NS) {
         *ctx.abort_flag = 1;
         if (atomicCAS(ctx.status, 0, -6 /* FCP_ERR_TIMEOUT */) == 0) {
           ctx.status[1] = where;
@@ -79,6 +80,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
       }
     }
   }
+  return true;
 }
 
 // Same, for code that must stay warp-convergent (it is followed by .sync.aligned instructions):
@@ -174,6 +176,53 @@ __device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr, uint32_t lbo_byte
   return d;
 }
 
+// The same descriptor split into its two 32-bit words, so that issue loops only add a byte offset to
+// the low word (start address field) instead of rebuilding all 64 bits per instruction.
+__device__ __forceinline__ uint32_t sdesc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__device__ __forceinline__ constexpr uint32_t sdesc_hi(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
+}
+__device__ __forceinline__ uint64_t sdesc_pack(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
+}
+
+// One 128 x N x (16*KSTEPS) product.  Fully unrolled with the descriptor offsets folded into
+// constants: a single thread issues these, and a rolled loop's dependent integer arithmetic (about
+// 85 clocks per trip) would be slower than the 64 clocks a 128x128x16 UMMA takes to execute.
+// K-major A and B tiles of [128][64]-element swizzled blocks: K step k lives in block k/4 at byte
+// offset (k%4)*32 of every row.
+template <int KSTEPS>
+__device__ __forceinline__ void umma_loop_kk(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
+  const uint32_t hi = sdesc_hi(1024), alo = sdesc_lo(a_addr, 16), blo = sdesc_lo(b_addr, 16);
+#pragma unroll
+  for (int k = 0; k < KSTEPS; ++k) {
+    const uint32_t off = (uint32_t)(k >> 2) * (16384u >> 4) + (uint32_t)(k & 3) * 2u;
+    umma_ss(d_tmem, sdesc_pack(alo + off, hi), sdesc_pack(blo + off, hi), idesc, k > 0 ? 1u : 0u);
+  }
+}
+// MN-major A and B (64-element blocks 16384 bytes apart): K step k is rows [16k, 16k+16) = +2048 bytes.
+__device__ __forceinline__ void umma_loop_mm(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
+  const uint32_t hi = sdesc_hi(1024), alo = sdesc_lo(a_addr, 16384), blo = sdesc_lo(b_addr, 16384);
+#pragma unroll
+  for (int k = 0; k < 8; ++k)
+    umma_ss(d_tmem, sdesc_pack(alo + k * 128u, hi), sdesc_pack(blo + k * 128u, hi), idesc, k > 0 ? 1u : 0u);
+}
+// A from TMEM (bf16 pairs, 8 columns per K step; with `split` the second four steps start at
+// column 64), MN-major B.  `acc` = accumulate into D from the first step on.
+__device__ __forceinline__ void umma_loop_ts(uint32_t d_tmem, uint32_t a_tmem, bool split, uint32_t b_addr, uint32_t idesc,
+                                             uint32_t acc) {
+  const uint32_t hi = sdesc_hi(1024), blo = sdesc_lo(b_addr, 16384);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t col = (split && k >= 4) ? 64u + 8u * (k - 4) : 8u * k;
+    umma_ts(d_tmem, a_tmem + col, sdesc_pack(blo + k * 128u, hi), idesc, (acc | (k > 0)) ? 1u : 0u);
+  }
+}
+
 // TMEM address = (lane << 16) | column.
 __device__ __forceinline__ uint32_t tmem_addr(uint32_t base, uint32_t lane, uint32_t col) {
   return base + (lane << 16) + col;
@@ -191,6 +240,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr)
       : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&r)[8]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+               : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(

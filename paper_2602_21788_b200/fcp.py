@@ -19,8 +19,8 @@ FCP_ERR_CUDA, FCP_ERR_TIMEOUT, FCP_ERR_NOT_UPLOADED = -5, -6, -7
 FCP_MAX_DEGREE = 64
 
 TABLES = dict(cu_seqlens=0, chunk_offset=1, chunk_bounds=2, pairs=3, items=4, slot_offset=5, slot_rows=6,
-              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10)
-_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4)
+              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11)
+_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, bwd_work=2)
 INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7)
 
 EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
