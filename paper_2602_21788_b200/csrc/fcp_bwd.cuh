@@ -472,25 +472,42 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_fence_after();
         if constexpr (DQ_T) {
           // thread = head-dim index, columns = queries: a warp adds 32 consecutive floats per query.
-          // A rolled loop over 16-query slices keeps this code small enough to stay in the
-          // instruction cache next to the math warps' loops.
-          float* dst = a.dq_acc + ((int64_t)q_row * a.hq + h) * D + row;
-          const int64_t stride = (int64_t)a.hq * D;
-#pragma unroll 1
-          for (int c16 = 0; c16 < 8; ++c16) {
-            uint32_t qv[16];
-            tmem_ld16(t_dq + c16 * 16, qv);
-            tc_wait_ld();
-            if (c16 == 7) {                     // the last slice is in registers: hand the columns back
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(BAR(B_DQEMPTY));
-            }
-            const int nv = q_valid - c16 * 16;
+          char* dst = reinterpret_cast<char*>(a.dq_acc + ((int64_t)q_row * a.hq + h) * D + row);
+          const int64_t stride = (int64_t)a.hq * D * 4;
+          if (q_valid == 128) {
+            // whole tile into registers, columns handed back at once, then the reductions: they are
+            // slow (L2 round trips) and must not sit between the tile and the issuer's next product
+            uint32_t qv[128];
 #pragma unroll
-            for (int c = 0; c < 16; ++c)
-              if (c < nv) red_add_f32(dst + c * stride, __uint_as_float(qv[c]));
-            dst += 16 * stride;
+            for (int c = 0; c < 4; ++c) tmem_ld32(t_dq + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&qv[c * 32]));
+            tc_wait_ld();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(BAR(B_DQEMPTY));
+#pragma unroll
+            for (int c = 0; c < 128; ++c) {
+              red_add_f32(reinterpret_cast<float*>(dst), __uint_as_float(qv[c]));
+              dst += stride;
+            }
+          } else {
+            // ragged tile (end of a chunk): rolled loop over 16-query slices
+#pragma unroll 1
+            for (int c16 = 0; c16 < 8; ++c16) {
+              uint32_t qv[16];
+              tmem_ld16(t_dq + c16 * 16, qv);
+              tc_wait_ld();
+              if (c16 == 7) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(BAR(B_DQEMPTY));
+              }
+              const int nv = q_valid - c16 * 16;
+#pragma unroll
+              for (int c = 0; c < 16; ++c) {
+                if (c < nv) red_add_f32(reinterpret_cast<float*>(dst), __uint_as_float(qv[c]));
+                dst += stride;
+              }
+            }
           }
         } else {
           float* dst = a.dq_acc + (((int64_t)q_row + row) * a.hq + h) * D;
