@@ -179,6 +179,43 @@ int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* 
  * bounded wait inside a kernel expired).  Synchronises the device.                               */
 int fcp_last_device_status(const fcp_plan* plan, int32_t* status);
 
+/* ------------------------------------------------------------------------------------------
+ * fcp_attn_bwd_noalloc — device.  (The paper has no counterpart: this entry point exists for the
+ * way the library gets embedded, not for the method.)
+ *
+ * Same gradients as fcp_attn_bwd, for callers that are not allowed to allocate device memory when
+ * they reach the backward pass: code running under a framework whose memory pool must own every
+ * allocation, inside a region where cudaMalloc would synchronise the device or is forbidden
+ * outright, or on a device whose memory has already been handed out in full.  Such a caller cannot
+ * size and allocate the scratch buffer fcp_attn_bwd wants, and cannot call fcp_plan_upload either.
+ * Here the plan stays a host object (no fcp_plan_upload needed), and the work tables, status
+ * words and backward scratch all go into one fixed array of FCP_NOALLOC_MAX_BYTES that is part of
+ * the library image on every GPU that loads it.  The call itself performs only asynchronous
+ * copies, memsets and kernel launches on `stream`.
+ *
+ *   in : plan (from fcp_plan_blocks), q, k, v, o, d_o (bf16), lse (fp32): device, as for fcp_attn_bwd
+ *   out: dq, dk, dv (device bf16, every element written)
+ * Limits and rules
+ *   - fcp_noalloc_bytes_needed(plan) must not exceed FCP_NOALLOC_MAX_BYTES (roughly
+ *     4*T*hq*D bytes plus the tables); larger batches get FCP_ERR_WORKSPACE and must use
+ *     fcp_attn_bwd with their own scratch.
+ *   - The first call on each device looks up the array's device address and opts the kernel in to
+ *     its shared-memory size; make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents (the
+ *     function clears what has to start from zero).  Two calls that can overlap on the GPU, on
+ *     different streams or from different threads, corrupt each other: serialise them.
+ *   - The plan's host tables are read by the asynchronous copies: keep the plan alive until the
+ *     stream has passed this call.
+ * fcp_noalloc_device_status reads the status words of the last such call on the current device
+ * (synchronises the device; 0 = fine, FCP_ERR_TIMEOUT if a bounded wait in the kernel expired).
+ */
+#define FCP_NOALLOC_MAX_BYTES (32u << 20)
+int fcp_noalloc_bytes_needed(const fcp_plan* plan, int64_t* bytes);
+int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const void* k, const void* v,
+                         const void* o, const void* d_o, const float* lse, void* dq, void* dk,
+                         void* dv, void* stream);
+int fcp_noalloc_device_status(int32_t* status);
+
 /* Kernel timing for benchmarks.  fcp_plan_set_profiling(plan, 1) makes every compute call record a
  * CUDA event pair around each of its kernels on the launching stream (a ring of the last 64 launches
  * per kind); fcp_plan_kernel_ms returns, after the caller has synchronised, the number of recorded

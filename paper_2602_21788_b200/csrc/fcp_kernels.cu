@@ -565,3 +565,161 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   FCP_CUDA_CHECK(cudaStreamSynchronize(st));
   return FCP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Backward pass for callers that must not allocate device memory
+// ---------------------------------------------------------------------------------------------
+// Everything the backward grid needs besides the caller's tensors lives in this one fixed array:
+// status words and work counter, the plan's work tables, and the scratch of fcp_attn_bwd (fp32 dQ
+// accumulator, delta and LSE rows).  Each GPU that loads the library carries the array until the
+// process exits.  In host code `g_noalloc_arena` is only a handle for the runtime's symbol calls,
+// never a device pointer: the address kernels may use comes from cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_noalloc_arena[FCP_NOALLOC_MAX_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_noalloc_ptr[kMaxDevices] = {};   // device address of the arena, per device
+int g_noalloc_sms[kMaxDevices] = {};
+
+// One-time set-up for the current device: arena address, SM count, shared-memory opt-in of the
+// backward kernel.  None of these allocates.
+int noalloc_setup(int dev) {
+  if (g_noalloc_ptr[dev]) return FCP_OK;
+  void* p = nullptr;
+  FCP_CUDA_CHECK(cudaGetSymbolAddress(&p, g_noalloc_arena));
+  int sms = 0, major = 0;
+  FCP_CUDA_CHECK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  FCP_CUDA_CHECK(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  if (major != 10) {
+    fcp_set_error("device %d is not sm_100: this library is built for sm_100a only", dev);
+    return FCP_ERR_CUDA;
+  }
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_bwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<64>::DYN_BYTES));
+  FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_bwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdSmem<128>::DYN_BYTES));
+  g_noalloc_sms[dev] = sms;
+  g_noalloc_ptr[dev] = (unsigned char*)p;
+  return FCP_OK;
+}
+}  // namespace
+
+extern "C" int fcp_noalloc_bytes_needed(const fcp_plan* plan, int64_t* bytes) {
+  if (!plan || !bytes) return FCP_ERR_INVALID_ARG;
+  int64_t scratch = 0;
+  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
+  *bytes = 256 + al((int64_t)plan->bwd_units.size() * 4) + al((int64_t)plan->bwd_qranges.size() * 4) +
+           al((int64_t)plan->bwd_work.size() * 4) + al(scratch);
+  return FCP_OK;
+}
+
+extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                                    const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* stream) {
+  if (!plan || !q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv) {
+    fcp_set_error("fcp_attn_bwd_noalloc: NULL argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  int64_t need = 0, scratch = 0;
+  fcp_noalloc_bytes_needed(plan, &need);
+  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
+  if (need > (int64_t)FCP_NOALLOC_MAX_BYTES) {
+    fcp_set_error("fcp_attn_bwd_noalloc: this batch needs %lld bytes of scratch, the built-in arena holds %lld; "
+                  "use fcp_attn_bwd with a caller-provided scratch buffer",
+                  (long long)need, (long long)FCP_NOALLOC_MAX_BYTES);
+    return FCP_ERR_WORKSPACE;
+  }
+  int dev = 0;
+  FCP_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) {
+    fcp_set_error("fcp_attn_bwd_noalloc: device index %d not supported", dev);
+    return FCP_ERR_UNSUPPORTED;
+  }
+  int rc = noalloc_setup(dev);
+  if (rc != FCP_OK) return rc;
+  unsigned char* base = g_noalloc_ptr[dev];
+  cudaStream_t st = (cudaStream_t)stream;
+  const fcp_params& P = plan->params;
+  const int64_t T = plan->T, D = P.head_dim;
+
+  // carve the arena: [status, counter | units | qranges | work | scratch]
+  int64_t off = 256;
+  int32_t* d_status = (int32_t*)base;
+  int32_t* d_units = (int32_t*)(base + off);    off += al((int64_t)plan->bwd_units.size() * 4);
+  int32_t* d_qranges = (int32_t*)(base + off);  off += al((int64_t)plan->bwd_qranges.size() * 4);
+  int32_t* d_work = (int32_t*)(base + off);     off += al((int64_t)plan->bwd_work.size() * 4);
+  unsigned char* d_scratch = base + off;
+
+  // the arena still holds the previous call's data: status, work counter and the dQ accumulator
+  // must start at zero; the tables are rewritten from the plan's host copy
+  FCP_CUDA_CHECK(cudaMemsetAsync(d_status, 0, 256, st));
+  FCP_CUDA_CHECK(cudaMemsetAsync(d_scratch, 0, (size_t)scratch, st));
+  if (!plan->bwd_units.empty())
+    FCP_CUDA_CHECK(cudaMemcpyAsync(d_units, plan->bwd_units.data(), plan->bwd_units.size() * 4, cudaMemcpyHostToDevice, st));
+  if (!plan->bwd_qranges.empty())
+    FCP_CUDA_CHECK(cudaMemcpyAsync(d_qranges, plan->bwd_qranges.data(), plan->bwd_qranges.size() * 4, cudaMemcpyHostToDevice, st));
+  if (!plan->bwd_work.empty())
+    FCP_CUDA_CHECK(cudaMemcpyAsync(d_work, plan->bwd_work.data(), plan->bwd_work.size() * 4, cudaMemcpyHostToDevice, st));
+
+  const int64_t tpad = bwd_tpad(T);
+  float* dq_acc = (float*)d_scratch;
+  float* delta_t = dq_acc + T * P.hq * D;
+  float* lse2_t = delta_t + tpad * P.hq;
+  {
+    const int64_t rows = T * P.hq;
+    const int64_t blocks = (rows * (D / 8) + 255) / 256;
+    if (D == 128)
+      fcp_delta_kernel<128><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
+                                                              tpad, P.scale, delta_t, lse2_t);
+    else
+      fcp_delta_kernel<64><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
+                                                             tpad, P.scale, delta_t, lse2_t);
+    FCP_CUDA_CHECK(cudaGetLastError());
+  }
+  CUtensorMap tq, tk, tv, tdo;
+  if ((rc = make_thd_map(&tq, q, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tk, k, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tv, v, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
+  if ((rc = make_thd_map(&tdo, d_o, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
+  BwdArgs a;
+  a.units = d_units;
+  a.qranges = d_qranges;
+  a.work = d_work;
+  a.n_work = (int32_t)(plan->bwd_work.size() / 2);
+  a.counter = d_status + 16;
+  a.hq = P.hq;
+  a.hkv = P.hkv;
+  a.T = T;
+  a.t_stride = tpad;
+  a.scale = P.scale;
+  a.scale_log2 = P.scale * 1.4426950408889634f;
+  a.delta_t = delta_t;
+  a.lse2_t = lse2_t;
+  a.dq_acc = dq_acc;
+  a.dk = (__nv_bfloat16*)dk;
+  a.dv = (__nv_bfloat16*)dv;
+  a.status = d_status;
+  const int grid = (int)std::min<int64_t>(a.n_work, g_noalloc_sms[dev]);
+  if (grid > 0) {
+    if (D == 128)
+      fcp_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
+    else
+      fcp_bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
+    FCP_CUDA_CHECK(cudaGetLastError());
+  }
+  const int64_t n8 = T * P.hq * D / 8;
+  const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)g_noalloc_sms[dev] * 16);
+  fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8);
+  FCP_CUDA_CHECK(cudaGetLastError());
+  return FCP_OK;
+}
+
+extern "C" int fcp_noalloc_device_status(int32_t* status) {
+  if (!status) return FCP_ERR_INVALID_ARG;
+  int dev = 0;
+  FCP_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices || !g_noalloc_ptr[dev]) {
+    fcp_set_error("fcp_noalloc_device_status: fcp_attn_bwd_noalloc has not run on this device");
+    return FCP_ERR_INVALID_ARG;
+  }
+  FCP_CUDA_CHECK(cudaDeviceSynchronize());
+  FCP_CUDA_CHECK(cudaMemcpy(status, g_noalloc_ptr[dev], 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return FCP_OK;
+}

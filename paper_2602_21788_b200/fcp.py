@@ -26,7 +26,8 @@ INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merg
 EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
            "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_lse_merge", "fcp_attn_bwd",
            "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
-           "fcp_plan_kernel_ms", "fcp_status_string",
+           "fcp_plan_kernel_ms", "fcp_noalloc_bytes_needed", "fcp_attn_bwd_noalloc", "fcp_noalloc_device_status",
+           "fcp_status_string",
            "fcp_last_error_message"]
 
 
@@ -74,6 +75,9 @@ def lib() -> C.CDLL:
     L.fcp_host_workspace_bytes.argtypes = [vp, i64p]
     L.fcp_attn_fwd_bwd_host.argtypes = [vp] * 11 + [C.c_int64, vp]
     L.fcp_last_device_status.argtypes = [vp, i32p]
+    L.fcp_noalloc_bytes_needed.argtypes = [vp, i64p]
+    L.fcp_attn_bwd_noalloc.argtypes = [vp] * 11
+    L.fcp_noalloc_device_status.argtypes = [i32p]
     L.fcp_status_string.argtypes = [C.c_int]
     L.fcp_status_string.restype = C.c_char_p
     L.fcp_last_error_message.restype = C.c_char_p
@@ -211,3 +215,25 @@ def fcp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, scratch, scratch_
 def fcp_attn_fwd_bwd_host(plan: Plan, q, k, v, d_o, o, lse, dq, dk, dv, workspace, workspace_bytes, stream=0):
     _check(lib().fcp_attn_fwd_bwd_host(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(d_o), _ptr(o), _ptr(lse), _ptr(dq),
                                        _ptr(dk), _ptr(dv), _ptr(workspace), int(workspace_bytes), C.c_void_p(stream)))
+
+
+FCP_NOALLOC_MAX_BYTES = 32 << 20
+
+
+def fcp_noalloc_bytes_needed(plan: Plan) -> int:
+    v = C.c_int64(0)
+    _check(lib().fcp_noalloc_bytes_needed(plan.handle, C.byref(v)))
+    return v.value
+
+
+def fcp_attn_bwd_noalloc(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, stream=0):
+    """Backward pass that allocates nothing: the plan need not be uploaded and no scratch is passed;
+    the library's built-in arena (FCP_NOALLOC_MAX_BYTES per GPU) holds tables and scratch."""
+    _check(lib().fcp_attn_bwd_noalloc(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq),
+                                      _ptr(dk), _ptr(dv), C.c_void_p(stream)))
+
+
+def fcp_noalloc_device_status():
+    st = np.zeros(4, dtype=np.int32)
+    _check(lib().fcp_noalloc_device_status(st.ctypes.data_as(C.POINTER(C.c_int32))))
+    return st
