@@ -3,19 +3,23 @@
 //
 // Work unit = (two adjacent 128-row Q tiles of one plan item, one query head).  Roles per CTA:
 //   warp 0        TMA producer: Q tiles and the K/V tile ring (128-byte swizzled boxes)
-//   warp 1        UMMA issuer:  S = Q K^T into TMEM, O += P V with P read from TMEM
-//   warps 2..5    softmax for Q tile 0 (one thread per query row), epilogue
-//   warps 6..9    softmax for Q tile 1
+//   warps 1, 2    UMMA issuers, one per Q tile: S = Q K^T into TMEM, O += P V with P read from TMEM
+//   warps 4..7    softmax for Q tile 0 (one thread per query row), epilogue
+//   warps 8..11   softmax for Q tile 1
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each (D = 128); bf16 P overwrites the
 // first 64 columns of its S.  While one tile's softmax runs on the CUDA cores the tensor core works
 // on the other tile, so the two Q tiles share every K/V tile that is staged.
+//
+// The softmax makes two passes over its S tile in TMEM (row maximum, then exponentials) in rolled
+// loops of 32 columns: TMEM reads are cheap, and the small loop bodies keep the kernel's code inside
+// the instruction cache, which matters more than the extra reads.
 #pragma once
 #include "fcp_plan.hpp"
 #include "sm100_ptx.cuh"
 
 namespace fcp {
 
-constexpr int FWD_THREADS = 320;
+constexpr int FWD_THREADS = 384;
 constexpr int FWD_KV_SLOTS = 4;
 
 template <int D>
@@ -71,13 +75,13 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(BAR(B_QFULL + i), 1);
       mbar_init(BAR(B_QEMPTY + i), 1);
       mbar_init(BAR(B_SFULL + i), 1);
-      mbar_init(BAR(B_PFULL + i), 128);
+      mbar_init(BAR(B_PFULL + i), 4);          // one elected lane per softmax warp
       mbar_init(BAR(B_OFINAL + i), 1);
-      mbar_init(BAR(B_OEMPTY + i), 128);
+      mbar_init(BAR(B_OEMPTY + i), 4);
     }
     for (int i = 0; i < FWD_KV_SLOTS; ++i) {
       mbar_init(BAR(B_KVFULL + i), 1);
-      mbar_init(BAR(B_KVEMPTY + i), 1);
+      mbar_init(BAR(B_KVEMPTY + i), 2);        // one commit from each issuer
     }
     fence_mbar_init();
     prefetch_tmap(&tm_q);
@@ -101,17 +105,20 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (lane == 0) {
       uint32_t kv_it = 0, qcnt[2] = {0, 0};
       bool ok = true;
+#pragma unroll 1
       for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
         const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
         const int h = a.head_begin + (int)(w % a.head_count);
         const int hk = h / g;
         const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
         const int q_row0 = __ldg(U + FU_Q_ROW0);
+#pragma unroll 1
         for (int s = 0; s < 2 && ok; ++s) {
           if (nt[s] == 0) continue;
           ok = mbar_wait(BAR(B_QEMPTY + s), (qcnt[s] & 1) ^ 1, wctx, 10 + s);
           if (!ok) break;
           mbar_expect_tx(BAR(B_QFULL + s), SM::Q_TILE_BYTES);
+#pragma unroll 1
           for (int kb = 0; kb < KBLK; ++kb)
             tma_load_3d(sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES + kb * BLK_BYTES, &tm_q, BAR(B_QFULL + s), kb * 64, h,
                         q_row0 + s * 128);
@@ -120,13 +127,16 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int n_max = max(nt[0], nt[1]);
         const int nr0 = __ldg(U + FU_NT_RANGE0);
         const int kv0 = __ldg(U + FU_KV0_BEGIN), kv1 = __ldg(U + FU_KV1_BEGIN);
+#pragma unroll 1
         for (int j = 0; j < n_max && ok; ++j) {
           const int row = j < nr0 ? kv0 + j * 128 : kv1 + (j - nr0) * 128;
+#pragma unroll 1
           for (int t = 0; t < 2; ++t) {   // t = 0: K tile, t = 1: V tile
             const uint32_t slot = kv_it % FWD_KV_SLOTS;
             ok = mbar_wait(BAR(B_KVEMPTY + slot), ((kv_it / FWD_KV_SLOTS) & 1) ^ 1, wctx, 12);
             if (!ok) break;
             mbar_expect_tx(BAR(B_KVFULL + slot), SM::KV_TILE_BYTES);
+#pragma unroll 1
             for (int kb = 0; kb < KBLK; ++kb)
               tma_load_3d(sbase + SM::KV_OFF + slot * SM::KV_TILE_BYTES + kb * BLK_BYTES, t == 0 ? &tm_k : &tm_v,
                           BAR(B_KVFULL + slot), kb * 64, hk, row);
@@ -135,81 +145,75 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
       }
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ UMMA issuer
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------------ UMMA issuers, one per Q tile
+    // A single thread cannot issue the 32 UMMAs of one K/V tile (two Q tiles) plus its waits and
+    // commits in the 2048 clocks they take to execute, so each Q tile has its own issuing thread;
+    // their products touch disjoint TMEM columns and only read the shared K/V tiles.
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = make_idesc(128, 128, 0, 0);
       constexpr uint32_t IDESC_PV = make_idesc(128, D, 0, 1);
-      uint32_t kv_it = 0, qcnt[2] = {0, 0}, pcnt[2] = {0, 0}, ocnt[2] = {0, 0};
+      const int s = warp - 1;
+      const uint32_t t_s = tmem + S_COL0 + s * 128, t_o = tmem + O_COL0 + s * 128;
+      const uint32_t q_addr = sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES;
+      uint32_t kv_it = 0, qcnt = 0, pcnt = 0, ocnt = 0;
       bool ok = true;
+#pragma unroll 1
       for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
         const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
-        const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
-        const int n_max = max(nt[0], nt[1]);
-        for (int s = 0; s < 2 && ok; ++s)
-          if (nt[s] > 0) {
-            ok = mbar_wait(BAR(B_QFULL + s), qcnt[s] & 1, wctx, 20 + s);
-            ++qcnt[s];
-          }
+        const int nts = __ldg(U + FU_NT_STAGE0 + s);
+        const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
+        if (nts > 0) {
+          ok = mbar_wait(BAR(B_QFULL + s), qcnt & 1, wctx, 20 + s);
+          ++qcnt;
+        }
+#pragma unroll 1
         for (int j = 0; j <= n_max && ok; ++j) {
           // ring positions: K_j at kv_it + 2j, V_{j-1} at kv_it + 2j - 1
           const uint32_t itK = kv_it + 2 * j, itV = kv_it + 2 * j - 1;
           const uint32_t slotK = itK % FWD_KV_SLOTS, slotV = itV % FWD_KV_SLOTS;
+          // Every slot is awaited and released by both issuers, whether or not their tile uses it:
+          // a release may only be counted in the phase of the load it answers.
           if (j >= 1) ok = mbar_wait(BAR(B_KVFULL + slotV), (itV / FWD_KV_SLOTS) & 1, wctx, 22);
           if (ok && j < n_max) ok = mbar_wait(BAR(B_KVFULL + slotK), (itK / FWD_KV_SLOTS) & 1, wctx, 23);
           if (!ok) break;
-          for (int s = 0; s < 2 && ok; ++s) {
-            if (j >= 1 && j - 1 < nt[s]) {
-              // O_s (+)= P_s(j-1) V_{j-1}
-              if (j == 1) {
-                ok = mbar_wait(BAR(B_OEMPTY + s), (ocnt[s] & 1) ^ 1, wctx, 24 + s);
-                ++ocnt[s];
-                if (!ok) break;
-              }
-              ok = mbar_wait(BAR(B_PFULL + s), pcnt[s] & 1, wctx, 26 + s);
-              ++pcnt[s];
-              if (!ok) break;
-              tc_fence_after();
-              const uint32_t vbase = sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES;
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {   // 128 keys = 8 steps of K = 16
-                const uint64_t bdesc = make_sdesc(vbase + k * 2048, BLK_BYTES, 1024);
-                umma_ts(tmem + O_COL0 + s * 128, tmem + S_COL0 + s * 128 + k * 8, bdesc, IDESC_PV,
-                        (j > 1 || k > 0) ? 1u : 0u);
-              }
-              if (j - 1 == nt[s] - 1) tc_commit(BAR(B_OFINAL + s));
+          if (j >= 1 && j - 1 < nts) {
+            // O_s (+)= P_s(j-1) V_{j-1}
+            if (j == 1) {
+              ok = mbar_wait(BAR(B_OEMPTY + s), (ocnt & 1) ^ 1, wctx, 24 + s);
+              ++ocnt;
             }
-            if (j < nt[s]) {
-              // S_s = Q_s K_j^T
-              tc_fence_after();
-              const uint32_t qbase = sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES;
-              const uint32_t kbase = sbase + SM::KV_OFF + slotK * SM::KV_TILE_BYTES;
-#pragma unroll
-              for (int k = 0; k < D / 16; ++k) {
-                const uint32_t off = (k / 4) * BLK_BYTES + (k % 4) * 32;
-                umma_ss(tmem + S_COL0 + s * 128, make_sdesc(qbase + off, 16, 1024), make_sdesc(kbase + off, 16, 1024),
-                        IDESC_QK, k > 0 ? 1u : 0u);
-              }
-              tc_commit(BAR(B_SFULL + s));
-              if (j == nt[s] - 1) tc_commit(BAR(B_QEMPTY + s));
-            }
+            if (ok) ok = mbar_wait(BAR(B_PFULL + s), pcnt & 1, wctx, 26 + s);
+            ++pcnt;
+            if (!ok) break;
+            tc_fence_after();
+            umma_loop_ts(t_o, t_s, false, sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES, IDESC_PV, j > 1 ? 1u : 0u);
+            if (j == nts) tc_commit(BAR(B_OFINAL + s));
           }
-          if (!ok) break;
+          if (j < nts) {
+            // S_s = Q_s K_j^T
+            tc_fence_after();
+            umma_loop_kk<D / 16>(t_s, q_addr, sbase + SM::KV_OFF + slotK * SM::KV_TILE_BYTES, IDESC_QK);
+            tc_commit(BAR(B_SFULL + s));
+            if (j == nts - 1) tc_commit(BAR(B_QEMPTY + s));
+          }
           if (j >= 1) tc_commit(BAR(B_KVEMPTY + slotV));
           if (j < n_max) tc_commit(BAR(B_KVEMPTY + slotK));
         }
         kv_it += 2 * n_max;
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax + epilogue
-    const int s = (warp - 2) >> 2;            // Q tile handled by this warp group
-    const int rb = warp & 3;                  // TMEM lane block this warp may access
+    const int s = (warp - 4) >> 2;            // Q tile handled by this warp group
+    const int rb = warp & 3;                  // TMEM lane quarter this warp may access
     const int row = rb * 32 + lane;
     const uint32_t t_s = tmem_addr(tmem, rb * 32, S_COL0 + s * 128);
     const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
+    const float c2 = a.scale_log2;
     uint32_t scnt = 0, ucnt = 0;
     bool ok = true;
+#pragma unroll 1
     for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
       const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
       const int hl = (int)(w % a.head_count);
@@ -219,36 +223,37 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int rows_s = min(128, __ldg(U + FU_Q_ROWS) - s * 128);
       const int q_pos = q_row0 + row;
       const int nr0 = __ldg(U + FU_NT_RANGE0);
-      const int kvb[2] = {__ldg(U + FU_KV0_BEGIN), __ldg(U + FU_KV1_BEGIN)};
-      const int kve[2] = {__ldg(U + FU_KV0_END), __ldg(U + FU_KV1_END)};
-      const int kvd[2] = {__ldg(U + FU_KV0_DIAG), __ldg(U + FU_KV1_DIAG)};
+      const int kvb0 = __ldg(U + FU_KV0_BEGIN), kvb1 = __ldg(U + FU_KV1_BEGIN);
+      const int kve0 = __ldg(U + FU_KV0_END), kve1 = __ldg(U + FU_KV1_END);
+      const int kvd0 = __ldg(U + FU_KV0_DIAG), kvd1 = __ldg(U + FU_KV1_DIAG);
       float m_ref = -INFINITY, l = 0.f;
+#pragma unroll 1
       for (int j = 0; j < nts && ok; ++j) {
-        const int r = j < nr0 ? 0 : 1;
-        const int ks = r == 0 ? kvb[0] + j * 128 : kvb[1] + (j - nr0) * 128;
-        int limit = kve[r] - ks;                              // valid columns of this tile for this row
-        if (kvd[r]) limit = min(limit, q_pos - ks + 1);
+        const bool r1 = j >= nr0;
+        const int ks = r1 ? kvb1 + (j - nr0) * 128 : kvb0 + j * 128;
+        int limit = (r1 ? kve1 : kve0) - ks;                  // valid columns of this tile for this row
+        if (r1 ? kvd1 : kvd0) limit = min(limit, q_pos - ks + 1);
+        const bool masked = __any_sync(0xffffffffu, limit < 128);
         ok = mbar_wait_warp(BAR(B_SFULL + s), scnt & 1, wctx, 30 + s);
         ++scnt;
         if (!ok) break;
         tc_fence_after();
-        uint32_t sv[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&sv[c * 32]));
-        tc_wait_ld();
+        // pass 1: row maximum
         float mx = -INFINITY;
-        if (__any_sync(0xffffffffu, limit < 128)) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t sv[32];
+          tmem_ld32(t_s + c * 32, sv);
+          tc_wait_ld();
+          if (masked) {
 #pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float x = c < limit ? __uint_as_float(sv[c]) : -INFINITY;
-            sv[c] = __float_as_uint(x);
-            mx = fmaxf(mx, x);
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, c * 32 + i < limit ? __uint_as_float(sv[i]) : -INFINITY);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
           }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 128; ++c) mx = fmaxf(mx, __uint_as_float(sv[c]));
         }
-        mx *= a.scale_log2;
+        mx *= c2;
         // Lazy reference maximum: O and l are only rescaled when the row maximum grew by more than
         // 2^8, so p <= 256 always and the result is exact up to rounding.
         const bool grow = mx > m_ref + 8.f;
@@ -257,26 +262,34 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const float f = grow ? ex2(m_ref - m_new) : 1.f;    // m_ref = -inf -> 0
           l *= f;
           if (j > 0) {
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-              uint32_t ov[32];
-              tmem_ld32(t_o + c * 32, ov);
+#pragma unroll 1
+            for (int c = 0; c < D / 16; ++c) {
+              uint32_t ov[16];
+              tmem_ld16(t_o + c * 16, ov);
               tc_wait_ld();
 #pragma unroll
-              for (int i = 0; i < 32; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
-              tmem_st32(t_o + c * 32, ov);
+              for (int i = 0; i < 16; ++i) ov[i] = __float_as_uint(__uint_as_float(ov[i]) * f);
+              tmem_st16(t_o + c * 16, ov);
             }
           }
           m_ref = m_new;
         }
+        // pass 2: exponentials, row sum, bf16 P over the S columns already consumed
         float sum = 0.f;
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 4; ++c) {
+          uint32_t sv[32];
+          tmem_ld32(t_s + c * 32, sv);
+          tc_wait_ld();
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const float p0 = ex2(fmaf(__uint_as_float(sv[c * 32 + 2 * i]), a.scale_log2, -m_ref));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[c * 32 + 2 * i + 1]), a.scale_log2, -m_ref));
+            float p0 = ex2(fmaf(__uint_as_float(sv[2 * i]), c2, -m_ref));
+            float p1 = ex2(fmaf(__uint_as_float(sv[2 * i + 1]), c2, -m_ref));
+            if (masked) {
+              p0 = c * 32 + 2 * i < limit ? p0 : 0.f;
+              p1 = c * 32 + 2 * i + 1 < limit ? p1 : 0.f;
+            }
             sum += p0 + p1;
             pk[i] = pack_bf16(p0, p1);
           }
@@ -285,7 +298,8 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         l += sum;
         tc_wait_st();
         tc_fence_before();
-        mbar_arrive(BAR(B_PFULL + s));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_PFULL + s));
       }
       if (!ok) break;
       // epilogue: normalised partial output + log-sum-exp
@@ -296,23 +310,23 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const float inv_l = 1.f / l;
       const int64_t prow = (int64_t)__ldg(U + FU_PART_ROW0) + s * 128 + row;
       float* op = a.o_partial + (prow * a.head_count + hl) * D;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t ov[32];
-        tmem_ld32(t_o + c * 32, ov);
+#pragma unroll 1
+      for (int c = 0; c < D / 16; ++c) {
+        uint32_t ov[16];
+        tmem_ld16(t_o + c * 16, ov);
         tc_wait_ld();
         if (row < rows_s) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 4) {
-            float4 v4 = make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
-                                    __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
-            *reinterpret_cast<float4*>(op + c * 32 + i) = v4;
-          }
+          for (int i = 0; i < 16; i += 4)
+            *reinterpret_cast<float4*>(op + c * 16 + i) =
+                make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
+                            __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
         }
       }
       if (row < rows_s) a.lse_partial[prow * a.head_count + hl] = (m_ref + log2f(l)) * 0.6931471805599453f;
       tc_fence_before();
-      mbar_arrive(BAR(B_OEMPTY + s));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_OEMPTY + s));
     }
   }
 
