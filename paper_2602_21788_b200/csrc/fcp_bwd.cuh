@@ -326,7 +326,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else if (warp < 4 + BWD_MATH_WARPS) {
     // ------------------------------------------------------------------ math warps: C1, C2
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 128;");
     const int rb = warp & 3;                    // TMEM lane quarter
     const int half = (warp - 4) >> 2;           // which 64 of the 128 query columns
     const int row = rb * 32 + lane;             // key row of S^T / dP^T
@@ -450,7 +450,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------------ drain warps: C3, dK/dV epilogue
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 144;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 176;");
     const int rb = warp & 3;
     const int row = rb * 32 + lane;             // TMEM lane: head-dim index of dQ^T (or query row), key row of dK/dV
     const uint32_t t_dq = tmem_addr(tmem, rb * 32, C_DP);

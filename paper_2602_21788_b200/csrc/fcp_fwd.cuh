@@ -238,19 +238,27 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         ++scnt;
         if (!ok) break;
         tc_fence_after();
-        // pass 1: row maximum
+        // pass 1: row maximum.  Two register buffers: the next 32 columns are in flight while the
+        // current ones are reduced.
         float mx = -INFINITY;
+        {
+          uint32_t sv[2][32];
+          tmem_ld32(t_s, sv[0]);
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t sv[32];
-          tmem_ld32(t_s + c * 32, sv);
-          tc_wait_ld();
-          if (masked) {
+          for (int c2i = 0; c2i < 2; ++c2i) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, c * 32 + i < limit ? __uint_as_float(sv[i]) : -INFINITY);
-          } else {
+            for (int b = 0; b < 2; ++b) {
+              const int c = c2i * 2 + b;
+              tc_wait_ld();
+              if (c < 3) tmem_ld32(t_s + (c + 1) * 32, sv[b ^ 1]);
+              if (masked) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[i]));
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, c * 32 + i < limit ? __uint_as_float(sv[b][i]) : -INFINITY);
+              } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[b][i]));
+              }
+            }
           }
         }
         mx *= c2;
@@ -276,24 +284,32 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         // pass 2: exponentials, row sum, bf16 P over the S columns already consumed
         float sum = 0.f;
+        {
+          uint32_t sv[2][32];
+          tmem_ld32(t_s, sv[0]);
 #pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          uint32_t sv[32];
-          tmem_ld32(t_s + c * 32, sv);
-          tc_wait_ld();
-          uint32_t pk[16];
+          for (int c2i = 0; c2i < 2; ++c2i) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0 = ex2(fmaf(__uint_as_float(sv[2 * i]), c2, -m_ref));
-            float p1 = ex2(fmaf(__uint_as_float(sv[2 * i + 1]), c2, -m_ref));
-            if (masked) {
-              p0 = c * 32 + 2 * i < limit ? p0 : 0.f;
-              p1 = c * 32 + 2 * i + 1 < limit ? p1 : 0.f;
+            for (int b = 0; b < 2; ++b) {
+              const int c = c2i * 2 + b;
+              tc_wait_ld();
+              if (c < 3) tmem_ld32(t_s + (c + 1) * 32, sv[b ^ 1]);
+              uint32_t pk[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                float p0 = ex2(fmaf(__uint_as_float(sv[b][2 * i]), c2, -m_ref));
+                float p1 = ex2(fmaf(__uint_as_float(sv[b][2 * i + 1]), c2, -m_ref));
+                if (masked) {
+                  p0 = c * 32 + 2 * i < limit ? p0 : 0.f;
+                  p1 = c * 32 + 2 * i + 1 < limit ? p1 : 0.f;
+                }
+                sum += p0 + p1;
+                pk[i] = pack_bf16(p0, p1);
+              }
+              tc_wait_ld();                       // the columns about to be overwritten lie below the ones in flight
+              tmem_st16(t_s + c * 16, pk);
             }
-            sum += p0 + p1;
-            pk[i] = pack_bf16(p0, p1);
           }
-          tmem_st16(t_s + c * 16, pk);
         }
         l += sum;
         tc_wait_st();
