@@ -282,9 +282,9 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             if (ok) ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, wctx, 122);
             if (!ok) break;
             tc_fence_after();
-            umma_loop_kk<D / 16>(tmem + C_S, kbase, qbase, IDESC_ST);        // T1: S^T = K Q^T
+            umma_loop_kk<D / 16>(true, tmem + C_S, kbase, qbase, IDESC_ST);        // T1: S^T = K Q^T
             tc_commit(BAR(B_SFULL));
-            umma_loop_kk<D / 16>(tmem + C_DP, vbase, dobase, IDESC_ST);      // T2: dP^T = V dO^T
+            umma_loop_kk<D / 16>(true, tmem + C_DP, vbase, dobase, IDESC_ST);      // T2: dP^T = V dO^T
             tc_commit(BAR(B_DPFULL));
           }
           // T3: dV += P^T dO
@@ -292,21 +292,21 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           if (ok && i == 0) ok = mbar_wait(BAR(B_ACCEMPTY), (n & 1) ^ 1, wctx, 124);
           if (!ok) break;
           tc_fence_after();
-          umma_loop_ts(tmem + C_DV, tmem + C_S, true, dobase, IDESC_ACC, i > 0 ? 1u : 0u);
+          umma_loop_ts(true, tmem + C_DV, tmem + C_S, true, dobase, IDESC_ACC, i > 0 ? 1u : 0u);
           // T1 of the next tile: S^T has been read by the math warps and P^T is consumed in order
           if (i + 1 < n_iter) {
             ok = mbar_wait(BAR(B_QDOFULL + st_next), ((it + 1) / BWD_QDO_STAGES) & 1, wctx, 126);
             if (!ok) break;
-            umma_loop_kk<D / 16>(tmem + C_S, kbase, sbase + SM::Q_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
+            umma_loop_kk<D / 16>(true, tmem + C_S, kbase, sbase + SM::Q_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_SFULL));
           }
           // T4: dK += dS^T Q ; T5: dQ tile
           ok = mbar_wait(BAR(B_DSFULL), it & 1, wctx, 125);
           if (!ok) break;
           tc_fence_after();
-          umma_loop_ts(tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
-          if (DQ_T) umma_loop_mm(tmem + C_DP, kbase, dsbase, IDESC_DQ);
-          else umma_loop_mm(tmem + C_DP, dsbase, kbase, IDESC_DQ);
+          umma_loop_ts(true, tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
+          if (DQ_T) umma_loop_mm(true, tmem + C_DP, kbase, dsbase, IDESC_DQ);
+          else umma_loop_mm(true, tmem + C_DP, dsbase, kbase, IDESC_DQ);
           tc_commit(BAR(B_DQFULL));
           tc_commit(BAR(B_QDOFREE + st));
           // T2 of the next tile once the drain warps have emptied the dQ tile
@@ -314,7 +314,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ok = mbar_wait(BAR(B_DQEMPTY), it & 1, wctx, 127);
             if (!ok) break;
             tc_fence_after();
-            umma_loop_kk<D / 16>(tmem + C_DP, vbase, sbase + SM::DO_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
+            umma_loop_kk<D / 16>(true, tmem + C_DP, vbase, sbase + SM::DO_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_DPFULL));
           }
         }

@@ -29,8 +29,8 @@ struct FwdSmem {
   static constexpr int Q_OFF = 0;
   static constexpr int KV_OFF = 2 * Q_TILE_BYTES;
   static constexpr int BAR_OFF = KV_OFF + FWD_KV_SLOTS * KV_TILE_BYTES;
-  // barriers: q_full[2] q_empty[2] kv_full[S] kv_empty[S] s_full[2] p_full[2] o_final[2] o_empty[2]
-  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 8;
+  // barriers: q_full[2] q_empty[2] kv_full[S] kv_empty[S] s_full[2] p_full[2] o_final[2] o_empty[2] turn[2]
+  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 10;
   static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;   // tmem base (4 B), abort flag (4 B)
   static constexpr int TOTAL = MISC_OFF + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;          // slack to align the base to 1024 B
@@ -62,7 +62,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t bar0 = sbase + SM::BAR_OFF;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   const int B_QFULL = 0, B_QEMPTY = 2, B_KVFULL = 4, B_KVEMPTY = 4 + FWD_KV_SLOTS,
-            B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6;
+            B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6, B_TURN = B_SFULL + 8;
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
   volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
   const WaitCtx wctx{abort_flag, a.status};
@@ -78,6 +78,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(BAR(B_PFULL + i), 4);          // one elected lane per softmax warp
       mbar_init(BAR(B_OFINAL + i), 1);
       mbar_init(BAR(B_OEMPTY + i), 4);
+      mbar_init(BAR(B_TURN + i), 4);
     }
     for (int i = 0; i < FWD_KV_SLOTS; ++i) {
       mbar_init(BAR(B_KVFULL + i), 1);
@@ -150,7 +151,8 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // A single thread cannot issue the 32 UMMAs of one K/V tile (two Q tiles) plus its waits and
     // commits in the 2048 clocks they take to execute, so each Q tile has its own issuing thread;
     // their products touch disjoint TMEM columns and only read the shared K/V tiles.
-    if (lane == 0) {
+    {
+      const bool leader = lane == 0;   // the whole warp walks the schedule; one lane issues
       constexpr uint32_t IDESC_QK = make_idesc(128, 128, 0, 0);
       constexpr uint32_t IDESC_PV = make_idesc(128, D, 0, 1);
       const int s = warp - 1;
@@ -164,7 +166,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int nts = __ldg(U + FU_NT_STAGE0 + s);
         const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
         if (nts > 0) {
-          ok = mbar_wait(BAR(B_QFULL + s), qcnt & 1, wctx, 20 + s);
+          ok = mbar_wait_warp(BAR(B_QFULL + s), qcnt & 1, wctx, 20 + s);
           ++qcnt;
         }
 #pragma unroll 1
@@ -174,31 +176,31 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const uint32_t slotK = itK % FWD_KV_SLOTS, slotV = itV % FWD_KV_SLOTS;
           // Every slot is awaited and released by both issuers, whether or not their tile uses it:
           // a release may only be counted in the phase of the load it answers.
-          if (j >= 1) ok = mbar_wait(BAR(B_KVFULL + slotV), (itV / FWD_KV_SLOTS) & 1, wctx, 22);
-          if (ok && j < n_max) ok = mbar_wait(BAR(B_KVFULL + slotK), (itK / FWD_KV_SLOTS) & 1, wctx, 23);
+          if (j >= 1) ok = mbar_wait_warp(BAR(B_KVFULL + slotV), (itV / FWD_KV_SLOTS) & 1, wctx, 22);
+          if (ok && j < n_max) ok = mbar_wait_warp(BAR(B_KVFULL + slotK), (itK / FWD_KV_SLOTS) & 1, wctx, 23);
           if (!ok) break;
           if (j >= 1 && j - 1 < nts) {
             // O_s (+)= P_s(j-1) V_{j-1}
             if (j == 1) {
-              ok = mbar_wait(BAR(B_OEMPTY + s), (ocnt & 1) ^ 1, wctx, 24 + s);
+              ok = mbar_wait_warp(BAR(B_OEMPTY + s), (ocnt & 1) ^ 1, wctx, 24 + s);
               ++ocnt;
             }
-            if (ok) ok = mbar_wait(BAR(B_PFULL + s), pcnt & 1, wctx, 26 + s);
+            if (ok) ok = mbar_wait_warp(BAR(B_PFULL + s), pcnt & 1, wctx, 26 + s);
             ++pcnt;
             if (!ok) break;
             tc_fence_after();
-            umma_loop_ts(t_o, t_s, false, sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES, IDESC_PV, j > 1 ? 1u : 0u);
-            if (j == nts) tc_commit(BAR(B_OFINAL + s));
+            umma_loop_ts(leader, t_o, t_s, false, sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES, IDESC_PV, j > 1 ? 1u : 0u);
+            if (j == nts) tc_commit_if(leader, BAR(B_OFINAL + s));
           }
           if (j < nts) {
             // S_s = Q_s K_j^T
             tc_fence_after();
-            umma_loop_kk<D / 16>(t_s, q_addr, sbase + SM::KV_OFF + slotK * SM::KV_TILE_BYTES, IDESC_QK);
-            tc_commit(BAR(B_SFULL + s));
-            if (j == nts - 1) tc_commit(BAR(B_QEMPTY + s));
+            umma_loop_kk<D / 16>(leader, t_s, q_addr, sbase + SM::KV_OFF + slotK * SM::KV_TILE_BYTES, IDESC_QK);
+            tc_commit_if(leader, BAR(B_SFULL + s));
+            if (j == nts - 1) tc_commit_if(leader, BAR(B_QEMPTY + s));
           }
-          if (j >= 1) tc_commit(BAR(B_KVEMPTY + slotV));
-          if (j < n_max) tc_commit(BAR(B_KVEMPTY + slotK));
+          if (j >= 1) tc_commit_if(leader, BAR(B_KVEMPTY + slotV));
+          if (j < n_max) tc_commit_if(leader, BAR(B_KVEMPTY + slotK));
         }
         kv_it += 2 * n_max;
       }
@@ -211,14 +213,14 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t t_s = tmem_addr(tmem, rb * 32, S_COL0 + s * 128);
     const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
     const float c2 = a.scale_log2;
-    uint32_t scnt = 0, ucnt = 0;
+    uint32_t scnt = 0, ucnt = 0, tcnt = 0;
     bool ok = true;
 #pragma unroll 1
     for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
       const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
       const int hl = (int)(w % a.head_count);
       const int nts = __ldg(U + FU_NT_STAGE0 + s);
-      if (nts == 0) continue;
+      const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
       const int q_row0 = __ldg(U + FU_Q_ROW0) + s * 128;
       const int rows_s = min(128, __ldg(U + FU_Q_ROWS) - s * 128);
       const int q_pos = q_row0 + row;
@@ -228,7 +230,18 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int kvd0 = __ldg(U + FU_KV0_DIAG), kvd1 = __ldg(U + FU_KV1_DIAG);
       float m_ref = -INFINITY, l = 0.f;
 #pragma unroll 1
-      for (int j = 0; j < nts && ok; ++j) {
+      for (int j = 0; j < n_max && ok; ++j) {
+        // The two softmax groups take turns at the exponentials (the MUFU pipe cannot serve both at
+        // full speed): tile 0 of K/V tile j, tile 1 of j, tile 0 of j+1, ...  While one group is in
+        // its exponentials the tensor core runs the other tile's products.  A group without work
+        // for this j only passes the turn on.
+        if (j >= nts) {
+          ok = mbar_wait_warp(BAR(B_TURN + s), (tcnt & 1) ^ (s ^ 1), wctx, 34 + s);
+          ++tcnt;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(BAR(B_TURN + (s ^ 1)));
+          continue;
+        }
         const bool r1 = j >= nr0;
         const int ks = r1 ? kvb1 + (j - nr0) * 128 : kvb0 + j * 128;
         int limit = (r1 ? kve1 : kve0) - ks;                  // valid columns of this tile for this row
@@ -240,7 +253,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         tc_fence_after();
         // pass 1: row maximum.  Two register buffers: the next 32 columns are in flight while the
         // current ones are reduced.
-        float mx = -INFINITY;
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;   // independent chains
         {
           uint32_t sv[2][32];
           tmem_ld32(t_s, sv[0]);
@@ -253,15 +266,20 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               if (c < 3) tmem_ld32(t_s + (c + 1) * 32, sv[b ^ 1]);
               if (masked) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, c * 32 + i < limit ? __uint_as_float(sv[b][i]) : -INFINITY);
-              } else {
+                for (int i = 0; i < 32; ++i)
+                  if (c * 32 + i >= limit) sv[b][i] = 0xff800000u;     // -inf
+              }
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sv[b][i]));
+              for (int i = 0; i < 32; i += 8) {
+                mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sv[b][i]), __uint_as_float(sv[b][i + 1])));
+                mx1 = fmaxf(mx1, fmaxf(__uint_as_float(sv[b][i + 2]), __uint_as_float(sv[b][i + 3])));
+                mx2 = fmaxf(mx2, fmaxf(__uint_as_float(sv[b][i + 4]), __uint_as_float(sv[b][i + 5])));
+                mx3 = fmaxf(mx3, fmaxf(__uint_as_float(sv[b][i + 6]), __uint_as_float(sv[b][i + 7])));
               }
             }
           }
         }
-        mx *= c2;
+        float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c2;
         // Lazy reference maximum: O and l are only rescaled when the row maximum grew by more than
         // 2^8, so p <= 256 always and the result is exact up to rounding.
         const bool grow = mx > m_ref + 8.f;
@@ -282,8 +300,11 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
           m_ref = m_new;
         }
+        ok = mbar_wait_warp(BAR(B_TURN + s), (tcnt & 1) ^ (s ^ 1), wctx, 34 + s);
+        ++tcnt;
+        if (!ok) break;
         // pass 2: exponentials, row sum, bf16 P over the S columns already consumed
-        float sum = 0.f;
+        float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
         {
           uint32_t sv[2][32];
           tmem_ld32(t_s, sv[0]);
@@ -303,7 +324,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
                   p0 = c * 32 + 2 * i < limit ? p0 : 0.f;
                   p1 = c * 32 + 2 * i + 1 < limit ? p1 : 0.f;
                 }
-                sum += p0 + p1;
+                if ((i & 3) == 0) sum0 += p0 + p1;
+                else if ((i & 3) == 1) sum1 += p0 + p1;
+                else if ((i & 3) == 2) sum2 += p0 + p1;
+                else sum3 += p0 + p1;
                 pk[i] = pack_bf16(p0, p1);
               }
               tc_wait_ld();                       // the columns about to be overwritten lie below the ones in flight
@@ -311,13 +335,16 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
           }
         }
-        l += sum;
+        l += (sum0 + sum1) + (sum2 + sum3);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_TURN + (s ^ 1)));
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(B_PFULL + s));
       }
       if (!ok) break;
+      if (nts == 0) continue;
       // epilogue: normalised partial output + log-sum-exp
       ok = mbar_wait_warp(BAR(B_OFINAL + s), ucnt & 1, wctx, 32 + s);
       ++ucnt;

@@ -195,32 +195,43 @@ __device__ __forceinline__ uint64_t sdesc_pack(uint32_t lo, uint32_t hi) {
 // 85 clocks per trip) would be slower than the 64 clocks a 128x128x16 UMMA takes to execute.
 // K-major A and B tiles of [128][64]-element swizzled blocks: K step k lives in block k/4 at byte
 // offset (k%4)*32 of every row.
+//
+// The helpers are called by a whole warp in uniform control flow; only `leader` (one lane) executes
+// the UMMA itself.  Keeping the descriptor arithmetic outside the divergent part lets the compiler
+// hold it in the warp-uniform datapath instead of re-deriving it in one lane's registers.
 template <int KSTEPS>
-__device__ __forceinline__ void umma_loop_kk(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
+__device__ __forceinline__ void umma_loop_kk(bool leader, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
   const uint32_t hi = sdesc_hi(1024), alo = sdesc_lo(a_addr, 16), blo = sdesc_lo(b_addr, 16);
 #pragma unroll
   for (int k = 0; k < KSTEPS; ++k) {
     const uint32_t off = (uint32_t)(k >> 2) * (16384u >> 4) + (uint32_t)(k & 3) * 2u;
-    umma_ss(d_tmem, sdesc_pack(alo + off, hi), sdesc_pack(blo + off, hi), idesc, k > 0 ? 1u : 0u);
+    const uint64_t ad = sdesc_pack(alo + off, hi), bd = sdesc_pack(blo + off, hi);
+    if (leader) umma_ss(d_tmem, ad, bd, idesc, k > 0 ? 1u : 0u);
   }
 }
 // MN-major A and B (64-element blocks 16384 bytes apart): K step k is rows [16k, 16k+16) = +2048 bytes.
-__device__ __forceinline__ void umma_loop_mm(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
+__device__ __forceinline__ void umma_loop_mm(bool leader, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc) {
   const uint32_t hi = sdesc_hi(1024), alo = sdesc_lo(a_addr, 16384), blo = sdesc_lo(b_addr, 16384);
 #pragma unroll
-  for (int k = 0; k < 8; ++k)
-    umma_ss(d_tmem, sdesc_pack(alo + k * 128u, hi), sdesc_pack(blo + k * 128u, hi), idesc, k > 0 ? 1u : 0u);
+  for (int k = 0; k < 8; ++k) {
+    const uint64_t ad = sdesc_pack(alo + k * 128u, hi), bd = sdesc_pack(blo + k * 128u, hi);
+    if (leader) umma_ss(d_tmem, ad, bd, idesc, k > 0 ? 1u : 0u);
+  }
 }
 // A from TMEM (bf16 pairs, 8 columns per K step; with `split` the second four steps start at
 // column 64), MN-major B.  `acc` = accumulate into D from the first step on.
-__device__ __forceinline__ void umma_loop_ts(uint32_t d_tmem, uint32_t a_tmem, bool split, uint32_t b_addr, uint32_t idesc,
-                                             uint32_t acc) {
+__device__ __forceinline__ void umma_loop_ts(bool leader, uint32_t d_tmem, uint32_t a_tmem, bool split, uint32_t b_addr,
+                                             uint32_t idesc, uint32_t acc) {
   const uint32_t hi = sdesc_hi(1024), blo = sdesc_lo(b_addr, 16384);
 #pragma unroll
   for (int k = 0; k < 8; ++k) {
     const uint32_t col = (split && k >= 4) ? 64u + 8u * (k - 4) : 8u * k;
-    umma_ts(d_tmem, a_tmem + col, sdesc_pack(blo + k * 128u, hi), idesc, (acc | (k > 0)) ? 1u : 0u);
+    const uint64_t bd = sdesc_pack(blo + k * 128u, hi);
+    if (leader) umma_ts(d_tmem, a_tmem + col, bd, idesc, (acc | (k > 0)) ? 1u : 0u);
   }
+}
+__device__ __forceinline__ void tc_commit_if(bool leader, uint32_t bar) {
+  if (leader) tc_commit(bar);
 }
 
 // TMEM address = (lane << 16) | column.
