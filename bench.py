@@ -117,7 +117,7 @@ class ClockSampler:
         self.samples, self.proc = [], None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.th = threading.Thread(target=self._read, daemon=True)
             self.th.start()
@@ -173,7 +173,7 @@ def run_ours(args, w):
         w = synth.make_workload(w.name, seed=args.seed + rank)
     q, k, v, do = w.tensors()
     t_plan0 = time.perf_counter()
-    ds = DeviceState(w, q, k, v, do)
+    ds = DeviceState(w, q, k, v, do, heads_per_pass=args.heads_per_pass or None)
     plan_ms = 1e3 * (time.perf_counter() - t_plan0)
     plan = ds.plan
 
@@ -224,7 +224,7 @@ def run_ours(args, w):
 
     # ---- end to end from pinned host buffers through the host entry point
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.no_e2e:
         T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
         pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()
         hq_, hk_, hv_, hdo_ = pin(q), pin(k), pin(v), pin(do)
@@ -264,8 +264,9 @@ def run_ours(args, w):
         return
 
     # ---- roofline of the dominant kernel (backward attention): algorithmic FLOPs = 2.5 x forward
+    passes = -(-w.hq // ds.hpp)
     bwd_ms = kern["attn_bwd"]["mean_ms"]
-    fwd_ms = kern["attn_fwd"]["mean_ms"]
+    fwd_ms = kern["attn_fwd"]["mean_ms"] * passes      # all head passes of one step
     bwd_flops = 2.5 * w.flops_fwd()
     achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12 if bwd_ms > 0 else None
     peak = peaks["bf16_sustained"]
@@ -277,7 +278,7 @@ def run_ours(args, w):
                 "frac_of_vendor_dense_bf16": achieved / NOMINAL_BF16_TFLOPS if achieved else None}
     R = plan.info("R")
     merge_bytes = R * w.hq * (4 * w.head_dim + 4) + w.total_tokens * w.hq * (2 * w.head_dim + 4)
-    mms = kern["lse_merge"]["mean_ms"]
+    mms = kern["lse_merge"]["mean_ms"] * passes
     merge = {"bound": "hbm", "achieved_gbs": merge_bytes / (mms * 1e-3) / 1e9 if mms > 0 else None,
              "peak_gbs": peaks["hbm_gbs"], "ms": mms}
 
@@ -288,7 +289,6 @@ def run_ours(args, w):
         cpu = {"value": fl / dt / 1e12, "unit": "TFLOPS", "cores": blas_threads(), "kind": "oracle",
                "sample": f"{desc}; {dt:.1f} s of fp64 numpy"}
 
-    passes = -(-w.hq // ds.hpp)
     line = {
         "metric": METRIC, "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
@@ -297,7 +297,7 @@ def run_ours(args, w):
                    "hkv": w.hkv, "head_dim": w.head_dim, "seed": args.seed, "sum_len_sq": w.sum_sq,
                    "cp_degrees": sorted(set(int(x) for x in w.cp_degrees)), "partial_rows": R,
                    "l2": "inputs larger than L2 (q alone is %d MB)" % (2 * w.total_tokens * w.hq * w.head_dim >> 20),
-                   "flops": "7 * sum(L^2) * hq * head_dim per step", "plan_ms_host": plan_ms},
+                   "flops": "7 * sum(L^2) * hq * head_dim per step", "plan_ms_host": plan_ms, "head_passes": passes},
         "frac_of_peak": {"measured_sustained": value / world / peaks["bf16_sustained"],
                          "measured_burst": value / world / peaks["bf16_burst"],
                          "vendor_dense_bf16": value / world / NOMINAL_BF16_TFLOPS},
@@ -312,13 +312,15 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_64k")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--heads-per-pass", type=int, default=0, help="query heads per forward pass (0 = all)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
