@@ -170,7 +170,9 @@ def run_ours(args, w):
     # each rank has its own batch: independent problems, no data-path collective
     if world > 1:
         from paper_2602_21788_b200 import synth
-        w = synth.make_workload(w.name, seed=args.seed + rank)
+        w = synth.make_workload(args.workload, seed=args.seed + rank)
+        if args.max_heads > 0:
+            w = synth.reduced(w, len_div=1, max_heads=args.max_heads)
     q, k, v, do = w.tensors()
     t_plan0 = time.perf_counter()
     ds = DeviceState(w, q, k, v, do, heads_per_pass=args.heads_per_pass or None)
@@ -321,11 +323,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--heads-per-pass", type=int, default=0, help="query heads per forward pass (0 = all)")
+    ap.add_argument("--max-heads", type=int, default=0,
+                    help="keep at most this many query heads (query:KV ratio kept); a small case for profiler captures, "
+                         "named <workload>_reduced in the output")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     from paper_2602_21788_b200 import synth
     w = synth.make_workload(args.workload, args.seed)
+    if args.max_heads > 0:
+        w = synth.reduced(w, len_div=1, max_heads=args.max_heads)
     if args.impl == "reference":
         run_reference(args, w)
     else:
