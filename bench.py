@@ -27,6 +27,27 @@ sys.path.insert(0, ROOT)
 METRIC = "fwd+bwd attention TFLOPS/GPU on packed varlen batches"
 NOMINAL_BF16_TFLOPS = 2250.0      # vendor's public dense BF16 figure, for context only
 
+# DRAM bytes (read + write) of one backward-kernel launch from an ncu capture of this command line, with the
+# digest of the kernel sources the counters were taken on: reported only while the sources still match.
+NCU_BWD_TRAFFIC = {"llama8b_64k": (2534531072 + 1358226944, "0bdca916265198a8")}
+
+
+def bwd_kernel_digest():
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(os.path.dirname(os.path.abspath(__file__)), "paper_2602_21788_b200", "csrc")
+    for f in ("fcp_bwd.cuh", "sm100_ptx.cuh"):
+        with open(os.path.join(csrc, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(w, args):
+    rec = NCU_BWD_TRAFFIC.get(w.name)
+    if rec is None or args.max_heads > 0 or args.seed != 0:
+        return None
+    return rec[0] if rec[1] == bwd_kernel_digest() else None
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -273,7 +294,7 @@ def run_ours(args, w):
     achieved = bwd_flops / (bwd_ms * 1e-3) / 1e12 if bwd_ms > 0 else None
     peak = peaks["bf16_sustained"]
     roofline = {"bound": "tensor", "kernel": "fcp_bwd_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak if achieved else None, "traffic": None,
+                "frac": achieved / peak if achieved else None, "traffic": ncu_traffic(w, args),
                 "peak_source": f"{peaks['source']} sustained bf16 (kernel timed inside a long step)",
                 "fwd_kernel": {"achieved": w.flops_fwd() / (fwd_ms * 1e-3) / 1e12 if fwd_ms > 0 else None, "ms": fwd_ms},
                 "frac_of_burst": achieved / peaks["bf16_burst"] if achieved else None,

@@ -272,50 +272,48 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int n_iter = __ldg(U + BU_COST) * g;
         ok = mbar_wait(BAR(B_KVFULL), n & 1, wctx, 120);
         if (!ok) break;
+        // Software pipeline over the unit's tiles: trip i issues T3, T4, T5 of tile i and T1, T2 of tile
+        // i + 1; trip -1 only starts the first tile.  `it` counts the tiles whose T1/T2 have been issued.
 #pragma unroll 1
-        for (int i = 0; i < n_iter && ok; ++i, ++it) {
-          const uint32_t st = it % BWD_QDO_STAGES, st_next = (it + 1) % BWD_QDO_STAGES;
+        for (int i = -1; i < n_iter && ok; ++i) {
+          const bool cur = i >= 0, next = i + 1 < n_iter;
+          const uint32_t st = (it + 1) % BWD_QDO_STAGES, st_next = it % BWD_QDO_STAGES;   // tile i is tile it - 1
           const uint32_t qbase = sbase + SM::Q_OFF + st * SM::TILE_BYTES, dobase = sbase + SM::DO_OFF + st * SM::TILE_BYTES;
-          if (i == 0) {
-            // first tile of the unit: nothing was issued ahead
-            ok = mbar_wait(BAR(B_QDOFULL + st), (it / BWD_QDO_STAGES) & 1, wctx, 121);
-            if (ok) ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, wctx, 122);
+          if (cur) {
+            // T3: dV += P^T dO
+            ok = mbar_wait(BAR(B_PFULL), (it - 1) & 1, wctx, 123);
+            if (ok && i == 0) ok = mbar_wait(BAR(B_ACCEMPTY), (n & 1) ^ 1, wctx, 124);
             if (!ok) break;
             tc_fence_after();
-            umma_loop_kk<D / 16>(true, tmem + C_S, kbase, qbase, IDESC_ST);        // T1: S^T = K Q^T
-            tc_commit(BAR(B_SFULL));
-            umma_loop_kk<D / 16>(true, tmem + C_DP, vbase, dobase, IDESC_ST);      // T2: dP^T = V dO^T
-            tc_commit(BAR(B_DPFULL));
+            umma_loop_ts(true, tmem + C_DV, tmem + C_S, true, dobase, IDESC_ACC, i > 0 ? 1u : 0u);
           }
-          // T3: dV += P^T dO
-          ok = mbar_wait(BAR(B_PFULL), it & 1, wctx, 123);
-          if (ok && i == 0) ok = mbar_wait(BAR(B_ACCEMPTY), (n & 1) ^ 1, wctx, 124);
-          if (!ok) break;
-          tc_fence_after();
-          umma_loop_ts(true, tmem + C_DV, tmem + C_S, true, dobase, IDESC_ACC, i > 0 ? 1u : 0u);
           // T1 of the next tile: S^T has been read by the math warps and P^T is consumed in order
-          if (i + 1 < n_iter) {
-            ok = mbar_wait(BAR(B_QDOFULL + st_next), ((it + 1) / BWD_QDO_STAGES) & 1, wctx, 126);
+          if (next) {
+            ok = mbar_wait(BAR(B_QDOFULL + st_next), (it / BWD_QDO_STAGES) & 1, wctx, 126);
             if (!ok) break;
+            tc_fence_after();
             umma_loop_kk<D / 16>(true, tmem + C_S, kbase, sbase + SM::Q_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_SFULL));
           }
-          // T4: dK += dS^T Q ; T5: dQ tile
-          ok = mbar_wait(BAR(B_DSFULL), it & 1, wctx, 125);
-          if (!ok) break;
-          tc_fence_after();
-          umma_loop_ts(true, tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
-          if (DQ_T) umma_loop_mm(true, tmem + C_DP, kbase, dsbase, IDESC_DQ);
-          else umma_loop_mm(true, tmem + C_DP, dsbase, kbase, IDESC_DQ);
-          tc_commit(BAR(B_DQFULL));
-          tc_commit(BAR(B_QDOFREE + st));
-          // T2 of the next tile once the drain warps have emptied the dQ tile
-          if (i + 1 < n_iter) {
-            ok = mbar_wait(BAR(B_DQEMPTY), it & 1, wctx, 127);
+          if (cur) {
+            // T4: dK += dS^T Q ; T5: dQ tile
+            ok = mbar_wait(BAR(B_DSFULL), (it - 1) & 1, wctx, 125);
+            if (!ok) break;
+            tc_fence_after();
+            umma_loop_ts(true, tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
+            if (DQ_T) umma_loop_mm(true, tmem + C_DP, kbase, dsbase, IDESC_DQ);
+            else umma_loop_mm(true, tmem + C_DP, dsbase, kbase, IDESC_DQ);
+            tc_commit(BAR(B_DQFULL));
+            tc_commit(BAR(B_QDOFREE + st));
+          }
+          // T2 of the next tile once the drain warps have emptied the dQ tile of the one before it
+          if (next) {
+            ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, wctx, 127);
             if (!ok) break;
             tc_fence_after();
             umma_loop_kk<D / 16>(true, tmem + C_DP, vbase, sbase + SM::DO_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_DPFULL));
+            ++it;
           }
         }
         if (!ok) break;
@@ -477,17 +475,27 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           if (q_valid == 128) {
             // whole tile into registers, columns handed back at once, then the reductions: they are
             // slow (L2 round trips) and must not sit between the tile and the issuer's next product
-            uint32_t qv[128];
+            uint32_t qa[64], qb[64];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(t_dq + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&qv[c * 32]));
+            for (int c = 0; c < 2; ++c) {
+              tmem_ld32(t_dq + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&qa[c * 32]));
+              tmem_ld32(t_dq + 64 + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&qb[c * 32]));
+            }
             tc_wait_ld();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR(B_DQEMPTY));
+            // two rolled trips of 64 reductions (the second half moves down in between): half the
+            // code of a fully unrolled tile, which matters more to the instruction cache than the moves
+#pragma unroll 1
+            for (int hlf = 0; hlf < 2; ++hlf) {
 #pragma unroll
-            for (int c = 0; c < 128; ++c) {
-              red_add_f32(reinterpret_cast<float*>(dst), __uint_as_float(qv[c]));
-              dst += stride;
+              for (int c = 0; c < 64; ++c) {
+                red_add_f32(reinterpret_cast<float*>(dst), __uint_as_float(qa[c]));
+                dst += stride;
+              }
+#pragma unroll
+              for (int c = 0; c < 64; ++c) qa[c] = qb[c];
             }
           } else {
             // ragged tile (end of a chunk): rolled loop over 16-query slices
@@ -565,10 +573,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   }
 
-  if (*abort_flag) {
-    const unsigned long long t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
-  }
+  wait_teardown(wctx);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -401,12 +401,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   }
 
   // ---------------------------------------------------------------------- teardown
-  if (*abort_flag) {
-    // A wait gave up: give copies and MMAs still in flight time to land before the CTA's shared
-    // and tensor memory are released.
-    const unsigned long long t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
-  }
+  wait_teardown(wctx);
   tc_fence_before();
   __syncthreads();
   if (warp == 1) {

@@ -20,6 +20,12 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   return t;
 }
 
+__device__ __forceinline__ uint32_t globaltimer_lo() {
+  uint32_t t;
+  asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
+  return t;
+}
+
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
@@ -53,34 +59,49 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Shared per-CTA abort word + global status word.  `abort_flag` lives in shared memory.
+// Shared per-CTA abort word + global status word.  `abort_flag` lives in shared memory: zero while
+// all is well, else 0x40000000 | the `where` code of the first wait that gave up.
 struct WaitCtx {
-  volatile int* abort_flag;   // shared memory, set by the first waiter that gives up
-  int* status;                // global: [0] status, [1] where, [2] block, [3] extra
+  volatile int* abort_flag;
+  int* status;                // global: [0] status, [1] where, [2] block, [3] reserved
 };
 
 // Bounded wait.  Returns false if the CTA is aborting (this waiter timed out, or another did).
+// The body is inlined at every wait site of the persistent kernels, so it is kept to a few
+// instructions: the slow path only looks at the clock and the abort word; the status words are
+// written once, by wait_teardown().
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, int where) {
-  uint32_t spins = 0;
-  unsigned long long t0 = 0;
+  uint32_t spins = 0, t0 = 0;
 #pragma unroll 1
   while (!mbar_try_wait(bar, parity)) {
-    if ((++spins & 1023u) == 0) {
-      if (*ctx.abort_flag) return false;
-      const unsigned long long now = globaltimer_ns();
-      if (t0 == 0) t0 = now;
-      if (now - t0 > FCP_WAIT_NS) {
-        *ctx.abort_flag = 1;
-        if (atomicCAS(ctx.status, 0, -6 /* FCP_ERR_TIMEOUT */) == 0) {
-          ctx.status[1] = where;
-          ctx.status[2] = (int)blockIdx.x;
-          ctx.status[3] = (int)threadIdx.x;
-        }
+    if ((++spins & 2047u) == 0) {
+      // low word of the nanosecond timer: differences are exact modulo 2^32 (4.29 s), enough for
+      // the 2 s limit as long as the clock is looked at more often than that
+      const uint32_t now = globaltimer_lo();
+      if (spins == 2048u) t0 = now;
+      const int flag = *ctx.abort_flag;
+      if (flag != 0 || now - t0 > (uint32_t)FCP_WAIT_NS) {
+        if (flag == 0) *ctx.abort_flag = 0x40000000 | where;
         return false;
       }
     }
   }
   return true;
+}
+
+// End of a persistent kernel, called by every thread before the CTA-wide barrier that precedes the
+// release of tensor memory.  If a wait gave up: record who (first CTA wins) and give copies and MMAs
+// still in flight time to land before the CTA's shared and tensor memory are released.
+__device__ __forceinline__ void wait_teardown(const WaitCtx& ctx) {
+  const int flag = *ctx.abort_flag;
+  if (flag == 0) return;
+  if (threadIdx.x == 0 && atomicCAS(ctx.status, 0, -6 /* FCP_ERR_TIMEOUT */) == 0) {
+    ctx.status[1] = flag & 0xFFFF;
+    ctx.status[2] = (int)blockIdx.x;
+    ctx.status[3] = 0;
+  }
+  const unsigned long long t0 = globaltimer_ns();
+  while (globaltimer_ns() - t0 < 2000000ull) __nanosleep(1000);
 }
 
 // Same, for code that must stay warp-convergent (it is followed by .sync.aligned instructions):
