@@ -274,30 +274,35 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (!ok) break;
         // Software pipeline over the unit's tiles: trip i issues T3, T4, T5 of tile i and T1, T2 of tile
         // i + 1; trip -1 only starts the first tile.  `it` counts the tiles whose T1/T2 have been issued.
+        // Each barrier is looked at (mbar_test) one UMMA batch before it is needed.
+        bool p_ready = false;
 #pragma unroll 1
         for (int i = -1; i < n_iter && ok; ++i) {
           const bool cur = i >= 0, next = i + 1 < n_iter;
           const uint32_t st = (it + 1) % BWD_QDO_STAGES, st_next = it % BWD_QDO_STAGES;   // tile i is tile it - 1
           const uint32_t qbase = sbase + SM::Q_OFF + st * SM::TILE_BYTES, dobase = sbase + SM::DO_OFF + st * SM::TILE_BYTES;
+          bool q_ready = false, ds_ready = false;
           if (cur) {
             // T3: dV += P^T dO
-            ok = mbar_wait(BAR(B_PFULL), (it - 1) & 1, wctx, 123);
+            if (!p_ready) ok = mbar_wait(BAR(B_PFULL), (it - 1) & 1, wctx, 123);
             if (ok && i == 0) ok = mbar_wait(BAR(B_ACCEMPTY), (n & 1) ^ 1, wctx, 124);
             if (!ok) break;
+            if (next) q_ready = mbar_test(BAR(B_QDOFULL + st_next), (it / BWD_QDO_STAGES) & 1);
             tc_fence_after();
             umma_loop_ts(true, tmem + C_DV, tmem + C_S, true, dobase, IDESC_ACC, i > 0 ? 1u : 0u);
           }
           // T1 of the next tile: S^T has been read by the math warps and P^T is consumed in order
           if (next) {
-            ok = mbar_wait(BAR(B_QDOFULL + st_next), (it / BWD_QDO_STAGES) & 1, wctx, 126);
+            if (!q_ready) ok = mbar_wait(BAR(B_QDOFULL + st_next), (it / BWD_QDO_STAGES) & 1, wctx, 126);
             if (!ok) break;
+            if (cur) ds_ready = mbar_test(BAR(B_DSFULL), (it - 1) & 1);
             tc_fence_after();
             umma_loop_kk<D / 16>(true, tmem + C_S, kbase, sbase + SM::Q_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_SFULL));
           }
           if (cur) {
             // T4: dK += dS^T Q ; T5: dQ tile
-            ok = mbar_wait(BAR(B_DSFULL), (it - 1) & 1, wctx, 125);
+            if (!ds_ready) ok = mbar_wait(BAR(B_DSFULL), (it - 1) & 1, wctx, 125);
             if (!ok) break;
             tc_fence_after();
             umma_loop_ts(true, tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
@@ -307,9 +312,11 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_commit(BAR(B_QDOFREE + st));
           }
           // T2 of the next tile once the drain warps have emptied the dQ tile of the one before it
+          p_ready = false;
           if (next) {
             ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, wctx, 127);
             if (!ok) break;
+            p_ready = mbar_test(BAR(B_PFULL), it & 1);
             tc_fence_after();
             umma_loop_kk<D / 16>(true, tmem + C_DP, vbase, sbase + SM::DO_OFF + st_next * SM::TILE_BYTES, IDESC_ST);
             tc_commit(BAR(B_DPFULL));
@@ -370,39 +377,46 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         ok = mbar_wait_warp(BAR(B_SFULL), it & 1, wctx, 130);
         if (!ok) break;
         tc_fence_after();
-        uint32_t pk[32];                        // P^T of this key row and column half, bf16 pairs
-#pragma unroll
-        for (int c = 0; c < 2; ++c) {
-          uint32_t sv[32];
-          tmem_ld32(t_s + c * 32, sv);
-          tc_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float4 l4 = *reinterpret_cast<const float4*>(s_lse + c * 32 + 4 * i);
-            const float p0 = ex2(fmaf(__uint_as_float(sv[4 * i]), a.scale_log2, -l4.x));
-            const float p1 = ex2(fmaf(__uint_as_float(sv[4 * i + 1]), a.scale_log2, -l4.y));
-            const float p2 = ex2(fmaf(__uint_as_float(sv[4 * i + 2]), a.scale_log2, -l4.z));
-            const float p3 = ex2(fmaf(__uint_as_float(sv[4 * i + 3]), a.scale_log2, -l4.w));
-            pk[c * 16 + 2 * i] = pack_bf16(p0, p1);
-            pk[c * 16 + 2 * i + 1] = pack_bf16(p2, p3);
-          }
-        }
+        // P^T of this key row and column half as bf16 pairs: pa = query columns [0,32), pb = [32,64).
+        // C1 and C2 run as two rolled trips of 32 columns; between the trips the pair arrays rotate
+        // (register arrays cannot be indexed by the trip), which halves the code of this loop.
+        uint32_t pa[16], pb[16] = {};
+        unsigned long long keep = ~0ull;
         if (need_mask) {
           // valid query columns of this key row, relative to this warp's half: [lo, hi).  Bit j of
           // `keep` = column j survives; applied to the packed pairs.
           const int hi = min(64, max(0, (row < kv_rows ? q_valid : 0) - half * 64));
           const int lo = min(64, max(0, (causal ? kv_row0 + row - q_row : 0) - half * 64));
-          const unsigned long long ones = ~0ull;
-          const unsigned long long keep = (hi > lo) ? ((hi == 64 ? ones : ((1ull << hi) - 1)) & ~((1ull << lo) - 1)) : 0ull;
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const uint32_t b = (uint32_t)(keep >> (2 * j)) & 3u;
-            pk[j] &= (b & 1u ? 0x0000ffffu : 0u) | (b & 2u ? 0xffff0000u : 0u);
-          }
+          keep = (hi > lo) ? ((hi == 64 ? ~0ull : ((1ull << hi) - 1)) & ~((1ull << lo) - 1)) : 0ull;
         }
+#pragma unroll 1
+        for (int c = 0; c < 2; ++c) {
+          uint32_t sv[32];
+          tmem_ld32(t_s + c * 32, sv);
 #pragma unroll
-        for (int c = 0; c < 2; ++c)
-          tmem_st16(t_s + c * 16, *reinterpret_cast<uint32_t(*)[16]>(&pk[c * 16]));   // over this warp's own, already loaded, columns
+          for (int j = 0; j < 16; ++j) pa[j] = pb[j];
+          tc_wait_ld();
+          const float* lse_c = s_lse + c * 32;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float4 l4 = *reinterpret_cast<const float4*>(lse_c + 4 * i);
+            const float p0 = ex2(fmaf(__uint_as_float(sv[4 * i]), a.scale_log2, -l4.x));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[4 * i + 1]), a.scale_log2, -l4.y));
+            const float p2 = ex2(fmaf(__uint_as_float(sv[4 * i + 2]), a.scale_log2, -l4.z));
+            const float p3 = ex2(fmaf(__uint_as_float(sv[4 * i + 3]), a.scale_log2, -l4.w));
+            pb[2 * i] = pack_bf16(p0, p1);
+            pb[2 * i + 1] = pack_bf16(p2, p3);
+          }
+          if (need_mask) {
+            const uint32_t k32 = (uint32_t)(keep >> (32 * c));
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const uint32_t b2 = (k32 >> (2 * j)) & 3u;
+              pb[j] &= (b2 & 1u ? 0x0000ffffu : 0u) | (b2 & 2u ? 0xffff0000u : 0u);
+            }
+          }
+          tmem_st16(t_s + c * 16, pb);            // over this warp's own, already loaded, columns
+        }
         tc_wait_st();
         tc_fence_before();
         __syncwarp();
@@ -411,23 +425,26 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         ok = mbar_wait_warp(BAR(B_DPFULL), it & 1, wctx, 131);
         if (!ok) break;
         tc_fence_after();
-#pragma unroll
+#pragma unroll 1
         for (int c = 0; c < 2; ++c) {
           uint32_t dv_[32];
           tmem_ld32(t_dp + c * 32, dv_);
           tc_wait_ld();
+          const float* delta_c = s_delta + c * 32;
           uint32_t out[16];
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const float4 d4 = *reinterpret_cast<const float4*>(s_delta + c * 32 + 4 * i);
-            const uint32_t pa = pk[c * 16 + 2 * i], pb = pk[c * 16 + 2 * i + 1];
-            const float d0 = __uint_as_float(pa << 16) * fmaf(__uint_as_float(dv_[4 * i]), a.scale, -d4.x);
-            const float d1 = __uint_as_float(pa & 0xffff0000u) * fmaf(__uint_as_float(dv_[4 * i + 1]), a.scale, -d4.y);
-            const float d2 = __uint_as_float(pb << 16) * fmaf(__uint_as_float(dv_[4 * i + 2]), a.scale, -d4.z);
-            const float d3 = __uint_as_float(pb & 0xffff0000u) * fmaf(__uint_as_float(dv_[4 * i + 3]), a.scale, -d4.w);
+            const float4 d4 = *reinterpret_cast<const float4*>(delta_c + 4 * i);
+            const uint32_t pp = pa[2 * i], pq = pa[2 * i + 1];
+            const float d0 = __uint_as_float(pp << 16) * fmaf(__uint_as_float(dv_[4 * i]), a.scale, -d4.x);
+            const float d1 = __uint_as_float(pp & 0xffff0000u) * fmaf(__uint_as_float(dv_[4 * i + 1]), a.scale, -d4.y);
+            const float d2 = __uint_as_float(pq << 16) * fmaf(__uint_as_float(dv_[4 * i + 2]), a.scale, -d4.z);
+            const float d3 = __uint_as_float(pq & 0xffff0000u) * fmaf(__uint_as_float(dv_[4 * i + 3]), a.scale, -d4.w);
             out[2 * i] = pack_bf16(d0, d1);
             out[2 * i + 1] = pack_bf16(d2, d3);
           }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) pa[j] = pb[j];
           tmem_st16(t_dp + c * 16, out);
           // the same 32 values -> shared memory, keys x queries with queries contiguous (an
           // MN-major operand of the dQ product): 4 x 16-byte chunks, 128-byte swizzle

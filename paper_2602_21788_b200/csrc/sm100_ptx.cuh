@@ -59,6 +59,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking look at a barrier phase.  An issuing thread sends this ahead of a batch of UMMAs for
+// the barrier it will need after the batch: the answer travels while the batch is issued, and the
+// blocking wait (whose round trip through a busy memory pipe costs hundreds of clocks even when the
+// phase completed long ago) is skipped if it was already there.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 // Shared per-CTA abort word + global status word.  `abort_flag` lives in shared memory: zero while
 // all is well, else 0x40000000 | the `where` code of the first wait that gave up.
 struct WaitCtx {
