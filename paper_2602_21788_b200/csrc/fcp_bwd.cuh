@@ -7,10 +7,11 @@
 //   T2  dP^T = V dO^T                  (UMMA, smem x smem)      TMEM cols [128,256)
 //   C1  P^T  = exp2(S^T*c - lse2[q])   (CUDA cores, thread = key row x half of the queries), bf16 over S^T
 //   T3  dV  += P^T dO                  (UMMA, TMEM x smem)      TMEM cols [256,384)
-//   C2  dS^T = P^T o (dP^T*scale - delta[q]*scale)               bf16 over dP^T, and to smem
-//   T4  dK  += dS^T Q                  (UMMA, TMEM x smem)      TMEM cols [384,512)
+//   C2  dS^T = P^T o (dP^T*scale - delta[q]*scale)               bf16 to smem
 //   T5  dQ^T = K^T dS^T  (D = 128; rows = head-dim index)  or  dQ = dS K  (D = 64; rows = queries)
 //                                      (UMMA, smem x smem)      over dP^T
+//   T4  dK  += dS^T Q                  (UMMA, smem x smem)      TMEM cols [384,512); issued after T5 so
+//                                      that it runs while the drain warps read the dQ tile
 //   C3  dQ accumulator += tile         fp32 reductions to global memory (coalesced for D = 128)
 //
 // 16 warps: warp 0 TMA producer and work scheduler, warp 1 UMMA issuer (warps 2-3 idle), warps 4..11
@@ -301,14 +302,15 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             tc_commit(BAR(B_SFULL));
           }
           if (cur) {
-            // T4: dK += dS^T Q ; T5: dQ tile
+            // T5: dQ tile, handed to the drain warps at once; T4: dK += dS^T Q runs while they read it.
+            // Both take dS^T from shared memory (K-major A for T4, MN-major B for T5).
             if (!ds_ready) ok = mbar_wait(BAR(B_DSFULL), (it - 1) & 1, wctx, 125);
             if (!ok) break;
             tc_fence_after();
-            umma_loop_ts(true, tmem + C_DK, tmem + C_DP, true, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
             if (DQ_T) umma_loop_mm(true, tmem + C_DP, kbase, dsbase, IDESC_DQ);
             else umma_loop_mm(true, tmem + C_DP, dsbase, kbase, IDESC_DQ);
             tc_commit(BAR(B_DQFULL));
+            umma_loop_km(true, tmem + C_DK, dsbase, qbase, IDESC_ACC, i > 0 ? 1u : 0u);
             tc_commit(BAR(B_QDOFREE + st));
           }
           // T2 of the next tile once the drain warps have emptied the dQ tile of the one before it
@@ -445,9 +447,8 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
 #pragma unroll
           for (int j = 0; j < 16; ++j) pa[j] = pb[j];
-          tmem_st16(t_dp + c * 16, out);
-          // the same 32 values -> shared memory, keys x queries with queries contiguous (an
-          // MN-major operand of the dQ product): 4 x 16-byte chunks, 128-byte swizzle
+          // 32 values -> shared memory, keys x queries with queries contiguous (the K-major A operand
+          // of the dK product and the MN-major B operand of the dQ product): 4 x 16-byte chunks, 128-byte swizzle
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             const int cc = c * 4 + ch;                          // 16-byte chunk within this half's 128-byte row
@@ -456,7 +457,6 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
         fence_proxy_async_smem();
-        tc_wait_st();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(B_DSFULL));
@@ -503,13 +503,18 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive(BAR(B_DQEMPTY));
             // two rolled trips of 64 reductions (the second half moves down in between): half the
-            // code of a fully unrolled tile, which matters more to the instruction cache than the moves
+            // code of a fully unrolled tile, which matters more to the instruction cache than the moves.
+            // The reductions are paced (a short sleep after every 16) so that they spread over the time
+            // a tile takes: sent back to back they keep the load/store queues of the SM full, and every
+            // barrier poll and shared-memory access of the other warps then waits behind them.  Measured:
+            // any pause that sums to 1.2-2 us per tile gives the same gain; 3 us makes this warp the bound.
 #pragma unroll 1
             for (int hlf = 0; hlf < 2; ++hlf) {
 #pragma unroll
               for (int c = 0; c < 64; ++c) {
                 red_add_f32(reinterpret_cast<float*>(dst), __uint_as_float(qa[c]));
                 dst += stride;
+                if ((c & 15) == 15) __nanosleep(200);
               }
 #pragma unroll
               for (int c = 0; c < 64; ++c) qa[c] = qb[c];

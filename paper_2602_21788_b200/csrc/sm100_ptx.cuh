@@ -253,6 +253,18 @@ __device__ __forceinline__ void umma_loop_mm(bool leader, uint32_t d_tmem, uint3
     if (leader) umma_ss(d_tmem, ad, bd, idesc, k > 0 ? 1u : 0u);
   }
 }
+// K-major A ([128][64]-element swizzled blocks, as in umma_loop_kk) and MN-major B (as in
+// umma_loop_mm); `acc` = accumulate into D from the first step on.
+__device__ __forceinline__ void umma_loop_km(bool leader, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, uint32_t idesc,
+                                             uint32_t acc) {
+  const uint32_t hi = sdesc_hi(1024), alo = sdesc_lo(a_addr, 16), blo = sdesc_lo(b_addr, 16384);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const uint32_t off = (uint32_t)(k >> 2) * (16384u >> 4) + (uint32_t)(k & 3) * 2u;
+    const uint64_t ad = sdesc_pack(alo + off, hi), bd = sdesc_pack(blo + k * 128u, hi);
+    if (leader) umma_ss(d_tmem, ad, bd, idesc, (acc | (k > 0)) ? 1u : 0u);
+  }
+}
 // A from TMEM (bf16 pairs, 8 columns per K step; with `split` the second four steps start at
 // column 64), MN-major B.  `acc` = accumulate into D from the first step on.
 __device__ __forceinline__ void umma_loop_ts(bool leader, uint32_t d_tmem, uint32_t a_tmem, bool split, uint32_t b_addr,
