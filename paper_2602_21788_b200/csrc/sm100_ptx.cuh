@@ -85,6 +85,9 @@ struct WaitCtx {
 // instructions: the slow path only looks at the clock and the abort word; the status words are
 // written once, by wait_teardown().
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const WaitCtx& ctx, int where) {
+  // A phase that completed earlier is seen by the non-blocking test in tens of clocks; try_wait, which
+  // may park the thread, was measured at 600-900 clocks on a busy SM even then.
+  if (mbar_test(bar, parity)) return true;
   uint32_t spins = 0, t0 = 0;
 #pragma unroll 1
   while (!mbar_try_wait(bar, parity)) {
