@@ -167,7 +167,9 @@ int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void*
  * runs fcp_attn_fwd (in head passes that fit the workspace), fcp_lse_merge and fcp_attn_bwd, and
  * copies o, lse, dq, dk, dv back.  `workspace` is a caller-owned DEVICE buffer of
  * `workspace_bytes` >= fcp_host_workspace_bytes(plan); host pointers should be pinned for the
- * copies to be asynchronous.  Synchronises `stream` before returning.
+ * copies to be asynchronous.  d_o comes in while the forward pass runs and o, lse go out while the
+ * backward pass runs (two internal streams, ordered after the work already queued on `stream`).
+ * Synchronises `stream` before returning; every output is complete then.
  */
 int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes);
 int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host,

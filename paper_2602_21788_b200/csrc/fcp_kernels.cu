@@ -541,10 +541,35 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   const int64_t T = plan->T, D = P.head_dim;
   char* w = (char*)workspace;
   cudaStream_t st = (cudaStream_t)stream;
+  // Copies that no kernel is waiting for run on two side streams: dO comes in while the forward
+  // pass runs, O and LSE go out while the backward pass runs.  Everything is ordered after the work
+  // already queued on `stream` and is complete when this call returns.
+  struct Side {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t qkv = nullptr, d_o = nullptr, fwd = nullptr, o_out = nullptr;
+    ~Side() {
+      if (qkv) cudaEventDestroy(qkv);
+      if (d_o) cudaEventDestroy(d_o);
+      if (fwd) cudaEventDestroy(fwd);
+      if (o_out) cudaEventDestroy(o_out);
+      if (in) cudaStreamDestroy(in);
+      if (out) cudaStreamDestroy(out);
+    }
+  } side;
+  FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.in, cudaStreamNonBlocking));
+  FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.out, cudaStreamNonBlocking));
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.qkv, cudaEventDisableTiming));
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.d_o, cudaEventDisableTiming));
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.fwd, cudaEventDisableTiming));
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.o_out, cudaEventDisableTiming));
+
   FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q, q_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, st));
   FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k, k_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
   FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v, v_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o, d_o_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, st));
+  FCP_CUDA_CHECK(cudaEventRecord(side.qkv, st));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.in, side.qkv, 0));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o, d_o_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, side.in));
+  FCP_CUDA_CHECK(cudaEventRecord(side.d_o, side.in));
   for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
     const int hc = std::min(L.heads_per_pass, P.hq - h0);
     if ((rc = fcp_attn_fwd(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part), st)) != FCP_OK)
@@ -552,16 +577,24 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
     if ((rc = fcp_lse_merge(plan, (float*)(w + L.o_part), (float*)(w + L.lse_part), h0, hc, w + L.o, nullptr, (float*)(w + L.lse), st)) != FCP_OK)
       return rc;
   }
+  FCP_CUDA_CHECK(cudaEventRecord(side.fwd, st));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.fwd, 0));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(o_host, w + L.o, T * P.hq * D * 2, cudaMemcpyDeviceToHost, side.out));
+  FCP_CUDA_CHECK(cudaMemcpyAsync(lse_host, w + L.lse, T * P.hq * 4, cudaMemcpyDeviceToHost, side.out));
+  FCP_CUDA_CHECK(cudaEventRecord(side.o_out, side.out));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.d_o, 0));
   int64_t scratch = 0;
   fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
   if ((rc = fcp_attn_bwd(plan, w + L.q, w + L.k, w + L.v, w + L.o, w + L.d_o, (float*)(w + L.lse), w + L.dq, w + L.dk,
-                         w + L.dv, w + L.scratch, scratch, st)) != FCP_OK)
+                         w + L.dv, w + L.scratch, scratch, st)) != FCP_OK) {
+    cudaStreamSynchronize(side.in);
+    cudaStreamSynchronize(side.out);
     return rc;
-  FCP_CUDA_CHECK(cudaMemcpyAsync(o_host, w + L.o, T * P.hq * D * 2, cudaMemcpyDeviceToHost, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(lse_host, w + L.lse, T * P.hq * 4, cudaMemcpyDeviceToHost, st));
+  }
   FCP_CUDA_CHECK(cudaMemcpyAsync(dq_host, w + L.dq, T * P.hq * D * 2, cudaMemcpyDeviceToHost, st));
   FCP_CUDA_CHECK(cudaMemcpyAsync(dk_host, w + L.dk, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
   FCP_CUDA_CHECK(cudaMemcpyAsync(dv_host, w + L.dv, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.o_out, 0));
   FCP_CUDA_CHECK(cudaStreamSynchronize(st));
   return FCP_OK;
 }

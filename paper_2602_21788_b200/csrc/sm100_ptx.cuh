@@ -341,20 +341,6 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// 2^x on the FMA pipe, for a share of the exponentials of a tile (the special-function unit does 16
-// per clock and SM and is the busiest unit of the softmax).  x is split into its nearest integer n
-// (the magic constant 1.5 * 2^23 leaves n in the low mantissa bits of t) and f = x - n in [-0.5, 0.5];
-// 2^f is a cubic fitted on that interval (largest relative error 7.5e-5, far below the bf16 rounding
-// the result receives), and n goes into the exponent field.  x <= -126 yields 2^-126; x must stay below 127.
-__device__ __forceinline__ float ex2_poly(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  float p = fmaf(0.05517161f, f, 0.24261111f);
-  p = fmaf(p, f, 0.69326097f);
-  p = fmaf(p, f, 0.99992806f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
