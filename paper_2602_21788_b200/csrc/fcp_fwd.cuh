@@ -4,23 +4,28 @@
 // Work unit = (two adjacent 128-row Q tiles of one plan item, one query head).  Roles per CTA:
 //   warp 0        TMA producer: Q tiles and the K/V tile ring (128-byte swizzled boxes)
 //   warps 1, 2    UMMA issuers, one per Q tile: S = Q K^T into TMEM, O += P V with P read from TMEM
-//   warps 4..11   softmax for Q tile 0 (two warps per 32 query rows, 64 key columns each), epilogue
-//   warps 12..19  softmax for Q tile 1
+//   warps 4..7    softmax for Q tile 0: one thread per query row, the whole 128-column row in registers
+//   warps 8..11   softmax for Q tile 1
+//   warps 12..15  epilogue for both tiles: normalise O, store the partial output and its log-sum-exp
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each (D = 128); bf16 P overwrites the
 // first 64 columns of its S.  While one tile's softmax runs on the CUDA cores the tensor core works
 // on the other tile, so the two Q tiles share every K/V tile that is staged.
 //
-// The softmax makes two passes over its S tile in TMEM (row maximum, then exponentials) in rolled
-// loops of 32 columns: TMEM reads are cheap, and the small loop bodies keep the kernel's code inside
-// the instruction cache, which matters more than the extra reads.
+// Registers are moved between the warp groups at start-up: a softmax thread holds a full row of S
+// (128 values), reads it from TMEM once, and needs no exchange with another thread for the row
+// maximum or the row sum; the producer/issuer and epilogue groups give up what they do not need.
 #pragma once
 #include "fcp_plan.hpp"
 #include "sm100_ptx.cuh"
 
 namespace fcp {
 
-constexpr int FWD_THREADS = 640;          // 4 control warps + 2 Q tiles x 8 softmax warps
+constexpr int FWD_THREADS = 512;          // 4 control warps + 2 x 4 softmax warps + 4 epilogue warps
 constexpr int FWD_KV_SLOTS = 4;
+// register budgets per thread of the three roles: 128 * 64 + 256 * 184 + 128 * 80 = 512 * 128
+#define FCP_FWD_REGS_CTRL "64"
+#define FCP_FWD_REGS_SOFTMAX "184"
+#define FCP_FWD_REGS_EPI "80"
 
 template <int D>
 struct FwdSmem {
@@ -30,10 +35,11 @@ struct FwdSmem {
   static constexpr int KV_OFF = 2 * Q_TILE_BYTES;
   static constexpr int BAR_OFF = KV_OFF + FWD_KV_SLOTS * KV_TILE_BYTES;
   // barriers: q_full[2] q_empty[2] kv_full[S] kv_empty[S] s_full[2] p_full[2] o_final[2] o_empty[2] turn[2]
-  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 10 + 8;   // + pair[8]
+  //           stat_full[2] stat_empty[2]
+  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 14;
   static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;   // tmem base (4 B), abort flag (4 B)
-  static constexpr int XCHG_OFF = MISC_OFF + 16;          // [2 parities][2 tiles][2 halves][128 rows] fp32
-  static constexpr int TOTAL = XCHG_OFF + 2 * 2 * 2 * 128 * 4;
+  static constexpr int STAT_OFF = MISC_OFF + 16;          // [2 tiles][row sum, reference maximum][128 rows] fp32
+  static constexpr int TOTAL = STAT_OFF + 2 * 2 * 128 * 4;
   static constexpr int DYN_BYTES = TOTAL + 1024;          // slack to align the base to 1024 B
 };
 
@@ -63,7 +69,8 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t bar0 = sbase + SM::BAR_OFF;
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   const int B_QFULL = 0, B_QEMPTY = 2, B_KVFULL = 4, B_KVEMPTY = 4 + FWD_KV_SLOTS,
-            B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6, B_TURN = B_SFULL + 8, B_PAIR = B_SFULL + 10;
+            B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6,
+            B_TURN = B_SFULL + 8, B_STATFULL = B_SFULL + 10, B_STATEMPTY = B_SFULL + 12;
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
   volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
   const WaitCtx wctx{abort_flag, a.status};
@@ -76,12 +83,13 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(BAR(B_QFULL + i), 1);
       mbar_init(BAR(B_QEMPTY + i), 1);
       mbar_init(BAR(B_SFULL + i), 1);
-      mbar_init(BAR(B_PFULL + i), 8);          // one elected lane per softmax warp
+      mbar_init(BAR(B_PFULL + i), 4);          // one elected lane per softmax warp
       mbar_init(BAR(B_OFINAL + i), 1);
-      mbar_init(BAR(B_OEMPTY + i), 8);
-      mbar_init(BAR(B_TURN + i), 8);
+      mbar_init(BAR(B_OEMPTY + i), 4);         // one elected lane per epilogue warp
+      mbar_init(BAR(B_TURN + i), 4);
+      mbar_init(BAR(B_STATFULL + i), 4);
+      mbar_init(BAR(B_STATEMPTY + i), 4);
     }
-    for (int i = 0; i < 8; ++i) mbar_init(BAR(B_PAIR + i), 2);   // the two warps that share 32 query rows
     for (int i = 0; i < FWD_KV_SLOTS; ++i) {
       mbar_init(BAR(B_KVFULL + i), 1);
       mbar_init(BAR(B_KVEMPTY + i), 2);        // one commit from each issuer
@@ -103,6 +111,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int64_t n_work = (int64_t)a.n_units * a.head_count;
   const int g = a.hq / a.hkv;
 
+  if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_CTRL ";");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -192,7 +201,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             ++pcnt;
             if (!ok) break;
             tc_fence_after();
-            umma_loop_ts(leader, t_o, t_s, true, sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES, IDESC_PV, j > 1 ? 1u : 0u);
+            umma_loop_ts(leader, t_o, t_s, false, sbase + SM::KV_OFF + slotV * SM::KV_TILE_BYTES, IDESC_PV, j > 1 ? 1u : 0u);
             if (j == nts) tc_commit_if(leader, BAR(B_OFINAL + s));
           }
           if (j < nts) {
@@ -208,48 +217,31 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         kv_it += 2 * n_max;
       }
     }
-  } else if (warp >= 4) {
-    // ------------------------------------------------------------------ softmax + epilogue
-    // Eight warps per Q tile: two per TMEM lane quarter, each thread one query row and half of the
-    // 128 key columns.  A single warp per scheduler cannot keep the MUFU pipe busy (about 11 clocks
-    // per warp-wide ex2 against 9 with two warps), and the shorter pass shortens the per-tile chain.
-    const int idx = warp - 4;
-    const int s = idx >> 3;                   // Q tile handled by this warp group
-    const int half = (idx >> 2) & 1;          // which 64 key columns
+  } else if (warp >= 4 && warp < 12) {
+    // ------------------------------------------------------------------ softmax
+    // Four warps per Q tile, one per TMEM lane quarter; a thread owns one query row and reads all 128
+    // scores of the current K/V tile into registers with one round of TMEM loads.
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 " FCP_FWD_REGS_SOFTMAX ";");
+    const int s = (warp - 4) >> 2;            // Q tile handled by this warp group
     const int rb = warp & 3;                  // TMEM lane quarter this warp may access
     const int row = rb * 32 + lane;
-    const uint32_t t_s = tmem_addr(tmem, rb * 32, S_COL0 + s * 128 + half * 64);   // own S columns; P goes over their first 32
-    const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128 + half * (D / 2));
-    const uint32_t pair_bar = BAR(B_PAIR + s * 4 + rb);
-    float* xchg = (float*)(smem + SM::XCHG_OFF);
-    auto xslot = [&](uint32_t parity, int h) -> float* { return xchg + ((parity * 2 + s) * 2 + h) * 128 + row; };
+    const uint32_t t_s = tmem_addr(tmem, rb * 32, S_COL0 + s * 128);   // P goes over the first 64 columns
+    const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
+    float* stat = (float*)(smem + SM::STAT_OFF) + s * 256;
     const float c2 = a.scale_log2;
-    uint32_t scnt = 0, ucnt = 0, tcnt = 0, xcnt = 0;
+    uint32_t scnt = 0, ucnt = 0, tcnt = 0;
     bool ok = true;
-    // exchange one float with the warp that owns the other half of the same rows
-    auto exchange = [&](float mine, float& other) -> bool {
-      *xslot(xcnt & 1, half) = mine;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(pair_bar);
-      const bool good = mbar_wait_warp(pair_bar, xcnt & 1, wctx, 36);
-      other = *xslot(xcnt & 1, half ^ 1);
-      ++xcnt;
-      return good;
-    };
 #pragma unroll 1
     for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
       const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
-      const int hl = (int)(w % a.head_count);
       const int nts = __ldg(U + FU_NT_STAGE0 + s);
       const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
-      const int q_row0 = __ldg(U + FU_Q_ROW0) + s * 128;
-      const int rows_s = min(128, __ldg(U + FU_Q_ROWS) - s * 128);
-      const int q_pos = q_row0 + row;
+      const int q_pos = __ldg(U + FU_Q_ROW0) + s * 128 + row;
       const int nr0 = __ldg(U + FU_NT_RANGE0);
       const int kvb0 = __ldg(U + FU_KV0_BEGIN), kvb1 = __ldg(U + FU_KV1_BEGIN);
       const int kve0 = __ldg(U + FU_KV0_END), kve1 = __ldg(U + FU_KV1_END);
       const int kvd0 = __ldg(U + FU_KV0_DIAG), kvd1 = __ldg(U + FU_KV1_DIAG);
-      float m_ref = -INFINITY, l = 0.f;       // l: this half's share of the row sum
+      float m_ref = -INFINITY, l = 0.f;
 #pragma unroll 1
       for (int j = 0; j < n_max && ok; ++j) {
         // The two softmax groups take turns at the exponentials (the MUFU pipe cannot serve both at
@@ -267,29 +259,27 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int ks = r1 ? kvb1 + (j - nr0) * 128 : kvb0 + j * 128;
         int limit = (r1 ? kve1 : kve0) - ks;                  // valid columns of this tile for this row
         if (r1 ? kvd1 : kvd0) limit = min(limit, q_pos - ks + 1);
-        limit -= half * 64;                                   // relative to this thread's 64 columns
-        const bool masked = __any_sync(0xffffffffu, limit < 64);
+        const bool masked = __any_sync(0xffffffffu, limit < 128);
         ok = mbar_wait_warp(BAR(B_SFULL + s), scnt & 1, wctx, 30 + s);
         ++scnt;
         if (!ok) break;
         tc_fence_after();
-        // pass 1: maximum over this thread's 64 columns (both loads in flight, independent chains),
-        // then the two warps of a row pair exchange their partial maxima.  (Reading the partner's
-        // columns instead would race with the partner's P, which it writes over its own S columns.)
+        uint32_t sv[4][32];
+#pragma unroll
+        for (int b = 0; b < 4; ++b) tmem_ld32(t_s + 32 * b, sv[b]);
+        tc_wait_ld();
+        if (masked) {
+#pragma unroll
+          for (int b = 0; b < 4; ++b)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (b * 32 + i >= limit) sv[b][i] = 0xff800000u;         // -inf
+        }
         float mx;
         {
-          uint32_t sv[2][32];
-          tmem_ld32(t_s, sv[0]);
-          tmem_ld32(t_s + 32, sv[1]);
-          tc_wait_ld();
           float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll
-          for (int b = 0; b < 2; ++b) {
-            if (masked) {
-#pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (b * 32 + i >= limit) sv[b][i] = 0xff800000u;       // -inf
-            }
+          for (int b = 0; b < 4; ++b)
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               mx0 = fmaxf(mx0, fmaxf(__uint_as_float(sv[b][i]), __uint_as_float(sv[b][i + 1])));
@@ -297,18 +287,11 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               mx2 = fmaxf(mx2, fmaxf(__uint_as_float(sv[b][i + 4]), __uint_as_float(sv[b][i + 5])));
               mx3 = fmaxf(mx3, fmaxf(__uint_as_float(sv[b][i + 6]), __uint_as_float(sv[b][i + 7])));
             }
-          }
-          mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-        }
-        {
-          float other;
-          ok = exchange(mx, other);
-          if (!ok) break;
-          mx = fmaxf(mx, other) * c2;                          // the row maximum over all 128 columns
+          mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * c2;
         }
         // Lazy reference maximum: O and l are only rescaled when the row maximum grew by more than
-        // 2^8, so p <= 256 always and the result is exact up to rounding.  Both halves of a row see
-        // the same maximum and take the same decision; each rescales its half of the O columns.
+        // 2^8, so p <= 256 always and the result is exact up to rounding.  The products issued so far
+        // have completed (S of this tile was committed after them), so O is at rest here.
         const bool grow = mx > m_ref + 8.f;
         if (__any_sync(0xffffffffu, grow)) {
           const float m_new = grow ? mx : m_ref;
@@ -316,7 +299,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           l *= f;
           if (j > 0) {
 #pragma unroll 1
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 16; ++c) {
               uint32_t ov[16];
               tmem_ld16(t_o + c * 16, ov);
               tc_wait_ld();
@@ -330,32 +313,22 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         ok = mbar_wait_warp(BAR(B_TURN + s), (tcnt & 1) ^ (s ^ 1), wctx, 34 + s);
         ++tcnt;
         if (!ok) break;
-        // pass 2: exponentials, row sum, bf16 P over the first 32 of this thread's own S columns
+        // exponentials, row sum, bf16 P over the first 64 columns of S (masked scores are -inf -> 0)
         float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-        {
-          uint32_t sv[2][32];
-          tmem_ld32(t_s, sv[0]);
-          tmem_ld32(t_s + 32, sv[1]);
-          tc_wait_ld();
 #pragma unroll
-          for (int b = 0; b < 2; ++b) {
-            uint32_t pk[16];
+        for (int b = 0; b < 4; ++b) {
+          uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              float p0 = ex2(fmaf(__uint_as_float(sv[b][2 * i]), c2, -m_ref));
-              float p1 = ex2(fmaf(__uint_as_float(sv[b][2 * i + 1]), c2, -m_ref));
-              if (masked) {
-                p0 = b * 32 + 2 * i < limit ? p0 : 0.f;
-                p1 = b * 32 + 2 * i + 1 < limit ? p1 : 0.f;
-              }
-              if ((i & 3) == 0) sum0 += p0 + p1;
-              else if ((i & 3) == 1) sum1 += p0 + p1;
-              else if ((i & 3) == 2) sum2 += p0 + p1;
-              else sum3 += p0 + p1;
-              pk[i] = pack_bf16(p0, p1);
-            }
-            tmem_st16(t_s + b * 16, pk);
+          for (int i = 0; i < 16; ++i) {
+            const float p0 = ex2(fmaf(__uint_as_float(sv[b][2 * i]), c2, -m_ref));
+            const float p1 = ex2(fmaf(__uint_as_float(sv[b][2 * i + 1]), c2, -m_ref));
+            if ((i & 3) == 0) sum0 += p0 + p1;
+            else if ((i & 3) == 1) sum1 += p0 + p1;
+            else if ((i & 3) == 2) sum2 += p0 + p1;
+            else sum3 += p0 + p1;
+            pk[i] = pack_bf16(p0, p1);
           }
+          tmem_st16(t_s + b * 16, pk);
         }
         l += (sum0 + sum1) + (sum2 + sum3);
         __syncwarp();
@@ -367,37 +340,67 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (!ok) break;
       if (nts == 0) continue;
-      // epilogue: normalised partial output + log-sum-exp; each half stores its D/2 columns
-      {
-        float other;
-        ok = exchange(l, other);
-        if (!ok) break;
-        l += other;
-      }
-      ok = mbar_wait_warp(BAR(B_OFINAL + s), ucnt & 1, wctx, 32 + s);
+      // hand the row sum and the reference maximum to the epilogue warps
+      ok = mbar_wait_warp(BAR(B_STATEMPTY + s), (ucnt & 1) ^ 1, wctx, 36 + s);
       ++ucnt;
       if (!ok) break;
-      tc_fence_after();
-      const float inv_l = 1.f / l;
-      const int64_t prow = (int64_t)__ldg(U + FU_PART_ROW0) + s * 128 + row;
-      float* op = a.o_partial + (prow * a.head_count + hl) * D + half * (D / 2);
-#pragma unroll 1
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t ov[16];
-        tmem_ld16(t_o + c * 16, ov);
-        tc_wait_ld();
-        if (row < rows_s) {
-#pragma unroll
-          for (int i = 0; i < 16; i += 4)
-            *reinterpret_cast<float4*>(op + c * 16 + i) =
-                make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
-                            __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
-        }
-      }
-      if (half == 0 && row < rows_s) a.lse_partial[prow * a.head_count + hl] = (m_ref + log2f(l)) * 0.6931471805599453f;
-      tc_fence_before();
+      stat[row] = l;
+      stat[128 + row] = m_ref;
       __syncwarp();
-      if (lane == 0) mbar_arrive(BAR(B_OEMPTY + s));
+      if (lane == 0) mbar_arrive(BAR(B_STATFULL + s));
+    }
+  } else if (warp >= 12) {
+    // ------------------------------------------------------------------ epilogue
+    // Normalised partial output + log-sum-exp of both Q tiles, while the softmax warps and the
+    // issuers already work on the next unit.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_EPI ";");
+    const int rb = warp & 3;
+    const int row = rb * 32 + lane;
+    uint32_t ecnt0 = 0, ecnt1 = 0;             // phases seen per Q tile
+    bool ok = true;
+#pragma unroll 1
+    for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
+      const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+      const int hl = (int)(w % a.head_count);
+      const int q_rows = __ldg(U + FU_Q_ROWS);
+      const int64_t prow0 = (int64_t)__ldg(U + FU_PART_ROW0);
+#pragma unroll 1
+      for (int s = 0; s < 2 && ok; ++s) {
+        if (__ldg(U + FU_NT_STAGE0 + s) == 0) continue;
+        const float* stat = (const float*)(smem + SM::STAT_OFF) + s * 256;
+        const uint32_t ph = (s ? ecnt1 : ecnt0) & 1;
+        if (s) ++ecnt1; else ++ecnt0;
+        ok = mbar_wait_warp(BAR(B_STATFULL + s), ph, wctx, 38 + s);
+        if (!ok) break;
+        const float l = stat[row], m_ref = stat[128 + row];
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_STATEMPTY + s));
+        ok = mbar_wait_warp(BAR(B_OFINAL + s), ph, wctx, 32 + s);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
+        const int rows_s = min(128, q_rows - s * 128);
+        const float inv_l = 1.f / l;
+        const int64_t prow = prow0 + s * 128 + row;
+        float* op = a.o_partial + (prow * a.head_count + hl) * D;
+#pragma unroll 1
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t ov[32];
+          tmem_ld32(t_o + c * 32, ov);
+          tc_wait_ld();
+          if (row < rows_s) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(op + c * 32 + i) =
+                  make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
+                              __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
+          }
+        }
+        if (row < rows_s) a.lse_partial[prow * a.head_count + hl] = (m_ref + log2f(l)) * 0.6931471805599453f;
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(B_OEMPTY + s));
+      }
     }
   }
 
