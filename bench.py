@@ -189,11 +189,9 @@ def run_ours(args, w):
     peaks = load_peaks()
 
     # each rank has its own batch: independent problems, no data-path collective
+    from paper_2602_21788_b200 import ranks
     if world > 1:
-        from paper_2602_21788_b200 import synth
-        w = synth.make_workload(args.workload, seed=args.seed + rank)
-        if args.max_heads > 0:
-            w = synth.reduced(w, len_div=1, max_heads=args.max_heads)
+        w = ranks.rank_workload(args.workload, args.seed, rank, world, args.max_heads)
     q, k, v, do = w.tensors()
     t_plan0 = time.perf_counter()
     ds = DeviceState(w, q, k, v, do, heads_per_pass=args.heads_per_pass or None)
@@ -233,17 +231,9 @@ def run_ours(args, w):
         kern[name] = {"launches": n, "mean_ms": kms}
     plan.set_profiling(False)
 
-    flops = w.flops_fwd_bwd()
-    if world > 1:
-        t = torch.tensor([ms, flops], dtype=torch.float64, device="cuda")
-        tmax = t.clone()
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        dist.all_reduce(t, op=dist.ReduceOp.SUM)
-        ms, flops_total = float(tmax[0]), float(t[1])
-    else:
-        flops_total = flops
+    ms, flops_total = ranks.aggregate(ms, w.flops_fwd_bwd(), "cuda")
     ms_per_step = ms / args.steps
-    value = flops_total / (ms_per_step * 1e-3) / 1e12
+    value = ranks.throughput_tflops(ms, args.steps, flops_total)
 
     # ---- end to end from pinned host buffers through the host entry point
     e2e = None
@@ -272,10 +262,7 @@ def run_ours(args, w):
         e1.record()
         barrier()
         e_ms = e0.elapsed_time(e1) / n_e2e
-        if world > 1:
-            t = torch.tensor([e_ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t[0])
+        e_ms, _ = ranks.aggregate(e_ms, 0.0, "cuda")
         h2d = 2 * (2 * T * hq * D + 2 * T * hkv * D)
         d2h = 2 * (2 * T * hq * D + 2 * T * hkv * D) + 4 * T * hq
         e2e = {"value": flops_total / (e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e_ms,
