@@ -199,7 +199,7 @@ def run_ours(args, w):
     plan = ds.plan
 
     def step():
-        ds.forward()
+        ds.forward(merged=True)
         ds.backward()
 
     def barrier():
@@ -287,7 +287,13 @@ def run_ours(args, w):
                 "frac_of_burst": achieved / peaks["bf16_burst"] if achieved else None,
                 "frac_of_vendor_dense_bf16": achieved / NOMINAL_BF16_TFLOPS if achieved else None}
     R = plan.info("R")
-    merge_bytes = R * w.hq * (4 * w.head_dim + 4) + w.total_tokens * w.hq * (2 * w.head_dim + 4)
+    # the merge launch only covers Q chunks with two or more slots (the forward kernel writes the others
+    # straight to the output): per token of such a chunk it reads every slot's partial row and writes one row
+    mu = plan.table("merge_units")[: plan.info("n_merge_multi")]
+    so = plan.table("slot_offset")
+    n_slots = (so[mu[:, 2] + 1] - so[mu[:, 2]]).astype(np.int64)
+    merge_tokens = int(mu[:, 1].sum())
+    merge_bytes = int((mu[:, 1] * n_slots).sum()) * w.hq * (4 * w.head_dim + 4) + merge_tokens * w.hq * (2 * w.head_dim + 4)
     mms = kern["lse_merge"]["mean_ms"] * passes
     merge = {"bound": "hbm", "achieved_gbs": merge_bytes / (mms * 1e-3) / 1e9 if mms > 0 else None,
              "peak_gbs": peaks["hbm_gbs"], "ms": mms}
@@ -305,7 +311,7 @@ def run_ours(args, w):
         "data": "synthetic",
         "config": {"workload": w.name, "tokens": w.total_tokens, "sequences": int(len(w.seqlens)), "hq": w.hq,
                    "hkv": w.hkv, "head_dim": w.head_dim, "seed": args.seed, "sum_len_sq": w.sum_sq,
-                   "cp_degrees": sorted(set(int(x) for x in w.cp_degrees)), "partial_rows": R,
+                   "cp_degrees": sorted(set(int(x) for x in w.cp_degrees)), "partial_rows": R, "merged_tokens": merge_tokens,
                    "l2": "inputs larger than L2 (q alone is %d MB)" % (2 * w.total_tokens * w.hq * w.head_dim >> 20),
                    "flops": "7 * sum(L^2) * hq * head_dim per step", "plan_ms_host": plan_ms, "head_passes": passes},
         "frac_of_peak": {"measured_sustained": value / world / peaks["bf16_sustained"],

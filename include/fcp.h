@@ -111,7 +111,8 @@ int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B
 int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count);
 
 /* Scalar facts about a plan: which in {0: T, 1: R (partial rows), 2: n_pairs, 3: n_items,
- * 4: n_fwd_units, 5: n_bwd_units, 6: n_merge_units, 7: B}.                                       */
+ * 4: n_fwd_units, 5: n_bwd_units, 6: n_merge_units, 7: B, 8: the leading merge units that belong
+ * to Q chunks with two or more slots (all that fcp_attn_fwd_merged has to merge)}.                */
 int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value);
 
 /* Bytes the caller must provide: o_partial = R*heads_per_pass*D*4, lse_partial = R*heads_per_pass*4,
@@ -136,6 +137,20 @@ int fcp_plan_destroy(fcp_plan* plan);
 int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v,
                  int32_t head_begin, int32_t head_count, float* o_partial, float* lse_partial,
                  void* stream);
+
+/* ------------------------------------------------------------------------------------------
+ * fcp_attn_fwd_merged — device.  fcp_attn_fwd followed by fcp_lse_merge in one call, for callers
+ * that do not need the partials of every item: Q chunks that have a single slot (every chunk of a
+ * sequence at degree 1, and the first chunk of any sequence) have nothing to merge, so their
+ * normalised partial is rounded to bf16 and written straight to o / lse, and only the chunks
+ * with two or more slots go through o_partial / lse_partial (same sizes as for fcp_attn_fwd) and
+ * the merge (Sec. 3.2: the merge re-associates the softmax sum; with one term it is the identity).
+ * o [T][hq][D] bf16 and lse [T][hq] fp32 are bit-identical to fcp_attn_fwd + fcp_lse_merge.
+ * After the call the partial rows of single-slot chunks are unspecified.  Asynchronous on `stream`.
+ */
+int fcp_attn_fwd_merged(const fcp_plan* plan, const void* q, const void* k, const void* v,
+                        int32_t head_begin, int32_t head_count, float* o_partial, float* lse_partial,
+                        void* o, float* lse, void* stream);
 
 /* ------------------------------------------------------------------------------------------
  * fcp_lse_merge — device.  Exact combination of the slots of every (token, head):

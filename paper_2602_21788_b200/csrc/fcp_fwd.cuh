@@ -50,6 +50,8 @@ struct FwdArgs {
   float scale_log2;       // softmax scale * log2(e)
   float* o_partial;       // [R][head_count][D]
   float* lse_partial;     // [R][head_count]
+  __nv_bfloat16* o_direct;   // [T][hq][D] or nullptr: final output of Q chunks that have a single slot
+  float* lse_direct;         // [T][hq]
   int32_t* status;        // [4]
 };
 
@@ -364,6 +366,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int hl = (int)(w % a.head_count);
       const int q_rows = __ldg(U + FU_Q_ROWS);
       const int64_t prow0 = (int64_t)__ldg(U + FU_PART_ROW0);
+      // A Q chunk with one slot has nothing to merge: its partial is the result, and goes straight to
+      // the output (rounded to bf16 exactly as the merge would round it) when the caller asks for that.
+      const bool direct = a.o_direct != nullptr && __ldg(U + FU_SINGLE_SLOT) != 0;
+      const int64_t trow0 = (int64_t)__ldg(U + FU_Q_ROW0);
 #pragma unroll 1
       for (int s = 0; s < 2 && ok; ++s) {
         if (__ldg(U + FU_NT_STAGE0 + s) == 0) continue;
@@ -381,22 +387,44 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
         const int rows_s = min(128, q_rows - s * 128);
         const float inv_l = 1.f / l;
-        const int64_t prow = prow0 + s * 128 + row;
-        float* op = a.o_partial + (prow * a.head_count + hl) * D;
+        const float lse_row = (m_ref + log2f(l)) * 0.6931471805599453f;
+        if (direct) {
+          const int64_t orow = (trow0 + s * 128 + row) * a.hq + a.head_begin + hl;
+          __nv_bfloat16* op = a.o_direct + orow * D;
 #pragma unroll 1
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t ov[32];
-          tmem_ld32(t_o + c * 32, ov);
-          tc_wait_ld();
-          if (row < rows_s) {
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(t_o + c * 32, ov);
+            tc_wait_ld();
+            if (row < rows_s) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-              *reinterpret_cast<float4*>(op + c * 32 + i) =
-                  make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
-                              __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
+              for (int i = 0; i < 32; i += 8)
+                *reinterpret_cast<uint4*>(op + c * 32 + i) =
+                    make_uint4(pack_bf16(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l),
+                               pack_bf16(__uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l),
+                               pack_bf16(__uint_as_float(ov[i + 4]) * inv_l, __uint_as_float(ov[i + 5]) * inv_l),
+                               pack_bf16(__uint_as_float(ov[i + 6]) * inv_l, __uint_as_float(ov[i + 7]) * inv_l));
+            }
           }
+          if (row < rows_s) a.lse_direct[orow] = lse_row;
+        } else {
+          const int64_t prow = prow0 + s * 128 + row;
+          float* op = a.o_partial + (prow * a.head_count + hl) * D;
+#pragma unroll 1
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t ov[32];
+            tmem_ld32(t_o + c * 32, ov);
+            tc_wait_ld();
+            if (row < rows_s) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4*>(op + c * 32 + i) =
+                    make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
+                                __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
+            }
+          }
+          if (row < rows_s) a.lse_partial[prow * a.head_count + hl] = lse_row;
         }
-        if (row < rows_s) a.lse_partial[prow * a.head_count + hl] = (m_ref + log2f(l)) * 0.6931471805599453f;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(BAR(B_OEMPTY + s));

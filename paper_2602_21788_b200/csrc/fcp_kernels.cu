@@ -327,8 +327,9 @@ static int check_heads(const fcp_plan* plan, int head_begin, int head_count) {
   return FCP_OK;
 }
 
-extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
-                            int32_t head_count, float* o_partial, float* lse_partial, void* stream) {
+namespace {
+int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin, int32_t head_count,
+               float* o_partial, float* lse_partial, void* o_direct, float* lse_direct, void* stream) {
   int rc = check_plan(plan);
   if (rc != FCP_OK) return rc;
   if (!q || !k || !v || !o_partial || !lse_partial) {
@@ -351,6 +352,8 @@ extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, 
   a.scale_log2 = P.scale * 1.4426950408889634f;
   a.o_partial = o_partial;
   a.lse_partial = lse_partial;
+  a.o_direct = (__nv_bfloat16*)o_direct;
+  a.lse_direct = lse_direct;
   a.status = plan->d_status;
   const int64_t n_work = (int64_t)a.n_units * head_count;
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
@@ -365,18 +368,9 @@ extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, 
   return FCP_OK;
 }
 
-extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
-                             int32_t head_begin, int32_t head_count, void* o, float* o_f32, float* lse,
-                             void* stream) {
-  int rc = check_plan(plan);
-  if (rc != FCP_OK) return rc;
-  if (!o_partial || !lse_partial || !o || !lse) {
-    fcp_set_error("fcp_lse_merge: NULL buffer");
-    return FCP_ERR_INVALID_ARG;
-  }
-  if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+int launch_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial, int32_t head_begin,
+                 int32_t head_count, void* o, float* o_f32, float* lse, int n_units, void* stream) {
   const fcp_params& P = plan->params;
-  const int n_units = (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W);
   if (n_units == 0) return FCP_OK;
   cudaStream_t st = (cudaStream_t)stream;
   ProfScope prof(plan, 1, st);
@@ -388,6 +382,38 @@ extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const
                                                   lse_partial, head_begin, head_count, P.hq, (__nv_bfloat16*)o, o_f32, lse);
   FCP_CUDA_CHECK(cudaGetLastError());
   return FCP_OK;
+}
+}  // namespace
+
+extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
+                            int32_t head_count, float* o_partial, float* lse_partial, void* stream) {
+  return launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, nullptr, nullptr, stream);
+}
+
+extern "C" int fcp_attn_fwd_merged(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
+                                   int32_t head_count, float* o_partial, float* lse_partial, void* o, float* lse,
+                                   void* stream) {
+  if (!o || !lse) {
+    fcp_set_error("fcp_attn_fwd_merged: NULL output");
+    return FCP_ERR_INVALID_ARG;
+  }
+  int rc = launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, o, lse, stream);
+  if (rc != FCP_OK) return rc;
+  return launch_merge(plan, o_partial, lse_partial, head_begin, head_count, o, nullptr, lse, plan->n_merge_multi, stream);
+}
+
+extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const float* lse_partial,
+                             int32_t head_begin, int32_t head_count, void* o, float* o_f32, float* lse,
+                             void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!o_partial || !lse_partial || !o || !lse) {
+    fcp_set_error("fcp_lse_merge: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+  return launch_merge(plan, o_partial, lse_partial, head_begin, head_count, o, o_f32, lse,
+                      (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W), stream);
 }
 
 extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
@@ -572,9 +598,8 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   FCP_CUDA_CHECK(cudaEventRecord(side.d_o, side.in));
   for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
     const int hc = std::min(L.heads_per_pass, P.hq - h0);
-    if ((rc = fcp_attn_fwd(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part), st)) != FCP_OK)
-      return rc;
-    if ((rc = fcp_lse_merge(plan, (float*)(w + L.o_part), (float*)(w + L.lse_part), h0, hc, w + L.o, nullptr, (float*)(w + L.lse), st)) != FCP_OK)
+    if ((rc = fcp_attn_fwd_merged(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part),
+                                  w + L.o, (float*)(w + L.lse), st)) != FCP_OK)
       return rc;
   }
   FCP_CUDA_CHECK(cudaEventRecord(side.fwd, st));

@@ -332,6 +332,10 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
       }
       u.f[FU_NT_RANGE0] = np == 2 ? nt_first : 0x7fffffff;
       u.f[FU_ITEM] = it;
+      {
+        const int ci = chunk_index0[b] + qc;   // a Q chunk with one slot needs no merge
+        u.f[FU_SINGLE_SLOT] = p->slot_offset[ci + 1] - p->slot_offset[ci] == 1;
+      }
       fus.push_back(u);
     }
   }
@@ -400,14 +404,23 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
         }
   }
 
-  // Merge: runs of up to FCP_MERGE_TOKENS tokens inside one chunk.
-  for (int b = 0; b < B; ++b) {
-    const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
-    for (int c = 0; c < 2 * cp_degrees[b]; ++c)
-      for (int32_t t = cbp[c]; t < cbp[c + 1]; t += FCP_MERGE_TOKENS) {
-        const int32_t rowm[4] = {t, std::min<int32_t>(FCP_MERGE_TOKENS, cbp[c + 1] - t), chunk_index0[b] + c, cbp[c]};
-        p->merge_units.insert(p->merge_units.end(), rowm, rowm + 4);
+  // Merge: runs of up to FCP_MERGE_TOKENS tokens inside one chunk.  Chunks with two or more slots
+  // come first: a forward pass that writes the single-slot chunks straight to the output only needs
+  // the first n_merge_multi units merged.
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int b = 0; b < B; ++b) {
+      const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+      for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
+        const int ci = chunk_index0[b] + c;
+        const bool single = p->slot_offset[ci + 1] - p->slot_offset[ci] <= 1;
+        if (single != (pass == 1)) continue;
+        for (int32_t t = cbp[c]; t < cbp[c + 1]; t += FCP_MERGE_TOKENS) {
+          const int32_t rowm[4] = {t, std::min<int32_t>(FCP_MERGE_TOKENS, cbp[c + 1] - t), ci, cbp[c]};
+          p->merge_units.insert(p->merge_units.end(), rowm, rowm + 4);
+        }
       }
+    }
+    if (pass == 0) p->n_merge_multi = (int32_t)(p->merge_units.size() / FCP_MERGE_UNIT_W);
   }
   *out = p;
   return FCP_OK;
@@ -447,6 +460,7 @@ extern "C" int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value
     case 5: *value = (int64_t)plan->bwd_units.size() / FCP_BWD_UNIT_W; break;
     case 6: *value = (int64_t)plan->merge_units.size() / FCP_MERGE_UNIT_W; break;
     case 7: *value = plan->B; break;
+    case 8: *value = plan->n_merge_multi; break;
     default: return FCP_ERR_INVALID_ARG;
   }
   return FCP_OK;

@@ -17,7 +17,7 @@ constexpr int FCP_MERGE_TOKENS = 16;   // tokens per merge work unit
 enum {
   FU_Q_ROW0 = 0, FU_Q_ROWS, FU_PART_ROW0, FU_N_RANGES,
   FU_KV0_BEGIN, FU_KV0_END, FU_KV0_DIAG, FU_KV1_BEGIN, FU_KV1_END, FU_KV1_DIAG,
-  FU_NT_STAGE0, FU_NT_STAGE1, FU_NT_RANGE0, FU_ITEM, FU_RSV0, FU_RSV1
+  FU_NT_STAGE0, FU_NT_STAGE1, FU_NT_RANGE0, FU_ITEM, FU_SINGLE_SLOT, FU_RSV1
 };
 // Field indices of a backward unit row and of a Q range row.
 enum { BU_KV_ROW0 = 0, BU_KV_ROWS, BU_FIRST_QRANGE, BU_N_QRANGES, BU_KV_TILE, BU_COST, BU_SEQ, BU_RSV };
@@ -29,6 +29,7 @@ struct fcp_plan {
   int32_t B = 0;
   int64_t T = 0;   // total tokens
   int64_t R = 0;   // rows of the partial buffers
+  int32_t n_merge_multi = 0;   // merge units of chunks with two or more slots (they come first in merge_units)
   std::vector<int32_t> cu_seqlens, chunk_offset, chunk_bounds, pairs, items, slot_offset, slot_rows;
   std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units, bwd_work;
 

@@ -21,10 +21,10 @@ FCP_MAX_DEGREE = 64
 TABLES = dict(cu_seqlens=0, chunk_offset=1, chunk_bounds=2, pairs=3, items=4, slot_offset=5, slot_rows=6,
               fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11)
 _TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, bwd_work=2)
-INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7)
+INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7, n_merge_multi=8)
 
 EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
-           "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_lse_merge", "fcp_attn_bwd",
+           "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_attn_fwd_merged", "fcp_lse_merge", "fcp_attn_bwd",
            "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
            "fcp_plan_kernel_ms", "fcp_noalloc_bytes_needed", "fcp_attn_bwd_noalloc", "fcp_noalloc_device_status",
            "fcp_status_string",
@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
     L.fcp_plan_destroy.argtypes = [vp]
     L.fcp_attn_fwd.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp]
     L.fcp_lse_merge.argtypes = [vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
+    L.fcp_attn_fwd_merged.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp, vp]
     L.fcp_plan_set_profiling.argtypes = [vp, C.c_int32]
     L.fcp_plan_kernel_ms.argtypes = [vp, C.c_int32, i32p, f32p]
     L.fcp_attn_bwd.argtypes = [vp] * 11 + [C.c_int64, vp]
@@ -199,6 +200,12 @@ def fcp_attn_fwd(plan: Plan, q, k, v, o_partial, lse_partial, head_begin=0, head
     hc = plan.hq - head_begin if head_count is None else head_count
     _check(lib().fcp_attn_fwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), int(head_begin), int(hc), _ptr(o_partial),
                               _ptr(lse_partial), C.c_void_p(stream)))
+
+
+def fcp_attn_fwd_merged(plan: Plan, q, k, v, o_partial, lse_partial, o, lse, head_begin=0, head_count=None, stream=0):
+    hc = plan.hq - head_begin if head_count is None else head_count
+    _check(lib().fcp_attn_fwd_merged(plan.handle, _ptr(q), _ptr(k), _ptr(v), int(head_begin), int(hc), _ptr(o_partial),
+                                     _ptr(lse_partial), _ptr(o), _ptr(lse), C.c_void_p(stream)))
 
 
 def fcp_lse_merge(plan: Plan, o_partial, lse_partial, o, lse, head_begin=0, head_count=None, stream=0, o_f32=None):

@@ -42,12 +42,18 @@ class DeviceState:
             self.scratch_bytes = self.plan.workspace_bytes(1)[2]
             self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device="cuda")
 
-    def forward(self, stream=None):
+    def forward(self, stream=None, merged=False):
+        """Forward over the plan + merge, in head passes.  `merged` uses the single call that writes
+        single-slot chunks straight to the output (no fp32 copy of the output, partials incomplete)."""
         st = (stream or torch.cuda.current_stream()).cuda_stream
         for h0 in range(0, self.w.hq, self.hpp):
             hc = min(self.hpp, self.w.hq - h0)
-            fcp.fcp_attn_fwd(self.plan, self.q, self.k, self.v, self.o_part, self.lse_part, h0, hc, st)
-            fcp.fcp_lse_merge(self.plan, self.o_part, self.lse_part, self.o, self.lse, h0, hc, st, o_f32=self.o_f32)
+            if merged:
+                fcp.fcp_attn_fwd_merged(self.plan, self.q, self.k, self.v, self.o_part, self.lse_part, self.o, self.lse,
+                                        h0, hc, st)
+            else:
+                fcp.fcp_attn_fwd(self.plan, self.q, self.k, self.v, self.o_part, self.lse_part, h0, hc, st)
+                fcp.fcp_lse_merge(self.plan, self.o_part, self.lse_part, self.o, self.lse, h0, hc, st, o_f32=self.o_f32)
 
     def backward(self, stream=None):
         st = (stream or torch.cuda.current_stream()).cuda_stream

@@ -127,6 +127,42 @@ def test_head_passes_give_the_same_result():
     assert np.array_equal(a["o"], b["o"]) and np.array_equal(a["lse"], b["lse"])
 
 
+MERGED_CASES = [
+    ([700, 300], [3, 2], 8, 2, 128, None),       # mixed single-slot (first chunks) and multi-slot chunks
+    ([3000, 129, 1], [1, 1, 1], 2, 1, 128, None),  # degree 1 everywhere: nothing left to merge
+    ([777, 64, 1500], [3, 1, 6], 4, 4, 64, 3),   # head_dim 64, head passes
+    ([1000], [7], 8, 1, 128, None),
+]
+
+
+@pytest.mark.parametrize("lens,degs,hq,hkv,D,hpp", MERGED_CASES)
+def test_merged_forward_is_bit_identical_to_forward_plus_merge(lens, degs, hq, hkv, D, hpp):
+    """fcp_attn_fwd_merged writes single-slot chunks straight to o / lse: same bits as the two calls,
+    and within the stated tolerances of the fp64 oracle."""
+    import torch
+    from paper_2602_21788_b200.runner import DeviceState, bf16_dev_to_f64
+    w = _wl(lens, degs, hq, hkv, D, seed=11)
+    q, k, v = w.tensors(with_do=False)
+    ds = DeviceState(w, q, k, v, None, heads_per_pass=hpp)
+    ds.forward()
+    torch.cuda.synchronize()
+    o_a, lse_a = ds.o.clone(), ds.lse.clone()
+    ds.o.fill_(float("nan"))
+    ds.lse.fill_(float("nan"))
+    ds.o_part.fill_(float("nan"))
+    ds.lse_part.fill_(float("nan"))
+    ds.forward(merged=True)
+    torch.cuda.synchronize()
+    ds.check_status()
+    assert torch.equal(ds.o.view(torch.int16), o_a.view(torch.int16))
+    assert torch.equal(ds.lse, lse_a)
+    f = synth.bf16_bits_to_f64
+    o_ref, lse_ref = A.attention_fwd_packed(f(q), f(k), f(v), w.cu_seqlens)
+    assert np.abs(ds.lse.cpu().numpy() - lse_ref).max() <= 1e-3
+    err = np.abs(bf16_dev_to_f64(ds.o) - o_ref)
+    assert err.mean() <= 1e-3 and (err <= 1e-2 + 2.0 ** -8 * np.abs(o_ref)).all()
+
+
 def test_forward_and_merge_are_bitwise_reproducible_and_backward_within_tolerance():
     from paper_2602_21788_b200.runner import run_fwd_bwd
     w = synth.make_workload("tiny", 1)
