@@ -190,6 +190,9 @@ def test_error_paths():
     with pytest.raises(fcp.FcpError) as e:
         fcp.fcp_plan_blocks([10], [0], 8, 2, 128)
     assert e.value.status == fcp.FCP_ERR_INVALID_ARG
+    with pytest.raises(fcp.FcpError) as e:                             # an empty batch is refused, not planned
+        fcp.fcp_plan_blocks([], [], 8, 2, 128)
+    assert e.value.status == fcp.FCP_ERR_INVALID_ARG
     with pytest.raises(fcp.FcpError) as e:
         fcp.fcp_plan_strategy([10], 4, 1.0, 1.0, 2.0, COEFFS[0])      # E <= M_ms
     assert e.value.status == fcp.FCP_ERR_INVALID_ARG

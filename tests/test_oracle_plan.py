@@ -185,10 +185,22 @@ def test_bfd_grouping_rules():
     assert dmin == [5]
 
 
+def _golden(name):
+    import os
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+
+
 def test_case_study_degree_mixes_use_the_whole_rank_budget():
-    """Table 6 reports mixes <8>x1,<6>x2,<4>x1,<2>x2,<1>x4 and <4>x2,<3>x4,<2>x6 on 32 ranks: the
-    allocator always spends exactly N ranks.  Reproduce the invariant on a skewed synthetic batch."""
-    assert 8 + 6 * 2 + 4 + 2 * 2 + 1 * 4 == 32 and 4 * 2 + 3 * 4 + 2 * 6 == 32
+    """Table 6 prints the CP-group mixes of two batches on 32 ranks (tests/golden/case_study_degree_mixes.txt):
+    every system spends exactly N ranks, and only FCP mixes degrees, non-powers-of-two among them.  The
+    allocator reproduces the invariant on a skewed synthetic batch."""
+    rows = [l.split() for l in open(_golden("case_study_degree_mixes.txt")) if l.strip() and not l.startswith("#")]
+    assert len(rows) == 6
+    for system, case, *mix in rows:
+        degs = [(int(a), int(b)) for a, b in (m.split("x") for m in mix)]
+        assert sum(d * n for d, n in degs) == 32, (system, case)
+        assert (len(degs) > 1) == (system == "FCP")
+    assert any(d & (d - 1) for s, c, *mix in rows if s == "FCP" for d in (int(m.split("x")[0]) for m in mix))
     rng = np.random.default_rng(3)
     lens = [int(x) for x in np.clip(rng.lognormal(8.0, 1.0, size=20), 256, 131072)]
     r = P.plan_strategy(lens, N=32, E=20000.0, M_token=1.0, M_ms=0.0, coeffs=COEFFS[0])
@@ -196,3 +208,20 @@ def test_case_study_degree_mixes_use_the_whole_rank_budget():
     assert all(d >= m for d, m in zip(r["d_group"], r["d_min"]))
     assert len(set(r["d_group"])) > 1                   # heterogeneous, incl. non-powers-of-two allowed
     assert P.plan_strategy([100000] * 5, N=4, E=1000.0, M_token=1.0, M_ms=0.0, coeffs=COEFFS[0]) is None
+
+
+def test_stored_plan_tables_match_the_oracle():
+    """tests/golden/plan_tables_small.json was written by tests/golden/make_plan_tables.py from this oracle: a
+    change in the reading of the plan (bounds, ring steps, slots, row order) shows up here."""
+    import json
+    for case in json.load(open(_golden("plan_tables_small.json"))):
+        ref = P.plan_blocks(case["lens"], case["degs"])
+        assert [int(x) for x in ref["chunk_bounds"]] == case["chunk_bounds"]
+        assert [[int(v) for v in p] for p in ref["pairs"]] == case["pairs"]
+        assert [[int(v) for v in i] for i in ref["items"]] == case["items"]
+        assert [[int(n), [int(v) for v in r]] for n, r in ref["chunk_slots"]] == case["chunk_slots"]
+        assert int(ref["n_partial_rows"]) == case["n_partial_rows"]
+        # closed forms that do not come from the oracle: d(2d+1) pairs for L >= 2d, chunk lengths sum to L
+        for b, (L, d) in enumerate(zip(case["lens"], case["degs"])):
+            if L >= 2 * d:
+                assert sum(1 for p in case["pairs"] if p[0] == b) == d * (2 * d + 1)
