@@ -179,11 +179,14 @@ int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void*
 
 /* ------------------------------------------------------------------------------------------
  * fcp_attn_fwd_bwd_host — the whole path from HOST buffers: copies q, k, v, d_o to the device,
- * runs fcp_attn_fwd (in head passes that fit the workspace), fcp_lse_merge and fcp_attn_bwd, and
- * copies o, lse, dq, dk, dv back.  `workspace` is a caller-owned DEVICE buffer of
- * `workspace_bytes` >= fcp_host_workspace_bytes(plan); host pointers should be pinned for the
- * copies to be asynchronous.  d_o comes in while the forward pass runs and o, lse go out while the
- * backward pass runs (two internal streams, ordered after the work already queued on `stream`).
+ * runs fcp_attn_fwd_merged (in head passes that fit the workspace) and fcp_attn_bwd, and copies
+ * o, lse, dq, dk, dv back.  `workspace` is a caller-owned DEVICE buffer of `workspace_bytes` >=
+ * fcp_host_workspace_bytes(plan); host pointers should be pinned for the copies to be asynchronous.
+ * The batch is cut into up to 8 runs of consecutive sequences (packed tensors are token-major, so a
+ * run is one contiguous slice of every tensor); the inputs of the next run come in and the results
+ * of the previous one go out while the kernels of the current run execute (two internal copy
+ * streams, ordered after the work already queued on `stream`).  The first call on a plan builds and
+ * uploads the plans of the runs (small device allocations, freed by fcp_plan_destroy).
  * Synchronises `stream` before returning; every output is complete then.
  */
 int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes);

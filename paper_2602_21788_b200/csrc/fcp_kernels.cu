@@ -284,6 +284,8 @@ extern "C" int fcp_plan_kernel_ms(const fcp_plan* plan, int32_t kind, int32_t* l
 
 extern "C" int fcp_plan_destroy(fcp_plan* plan) {
   if (!plan) return FCP_OK;
+  for (fcp_plan* g : plan->groups) fcp_plan_destroy(g);
+  plan->groups.clear();
   fcp_plan_set_profiling(plan, 0);
   if (plan->d_blob) cudaFree(plan->d_blob);
   delete plan;
@@ -296,6 +298,11 @@ extern "C" int fcp_last_device_status(const fcp_plan* plan, int32_t* status) {
   if (rc != FCP_OK) return rc;
   FCP_CUDA_CHECK(cudaDeviceSynchronize());
   FCP_CUDA_CHECK(cudaMemcpy(status, plan->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  // kernels launched by the host entry point report into the status words of its sequence groups
+  for (const fcp_plan* g : plan->groups) {
+    if (status[0] != 0) break;
+    FCP_CUDA_CHECK(cudaMemcpy(status, g->d_status, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  }
   return FCP_OK;
 }
 
@@ -547,6 +554,50 @@ extern "C" int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes) {
   return FCP_OK;
 }
 
+namespace {
+// Cuts the batch into runs of consecutive sequences of about equal token counts (at most 8 runs, at
+// least about 8192 tokens each) and plans each run on its own: packed tensors are token-major, so a run
+// is one contiguous slice of every tensor and can be copied, computed and copied back independently.
+int build_host_groups(const fcp_plan* plan, void* stream) {
+  if (!plan->groups.empty()) return FCP_OK;
+  const int B = plan->B;
+  const int64_t T = plan->T;
+  const int want = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(8, B), T / 8192));
+  std::vector<int32_t> lens(B), degs(B);
+  for (int b = 0; b < B; ++b) {
+    lens[b] = plan->cu_seqlens[b + 1] - plan->cu_seqlens[b];
+    degs[b] = (plan->chunk_offset[b + 1] - plan->chunk_offset[b] - 1) / 2;
+  }
+  std::vector<fcp_plan*> groups;
+  std::vector<int64_t> tok0;
+  int b0 = 0;
+  for (int g = 0; g < want && b0 < B; ++g) {
+    int b1 = b0 + 1;
+    if (g == want - 1) {
+      b1 = B;
+    } else {
+      const int64_t target = T * (g + 1) / want;
+      while (b1 < B - (want - 1 - g) && plan->cu_seqlens[b1] < target) ++b1;
+    }
+    fcp_plan* sub = nullptr;
+    int rc = fcp_plan_blocks(lens.data() + b0, degs.data() + b0, b1 - b0, &plan->params, &sub);
+    if (rc == FCP_OK) rc = fcp_plan_upload(sub, stream);
+    if (rc != FCP_OK) {
+      if (sub) fcp_plan_destroy(sub);
+      for (fcp_plan* x : groups) fcp_plan_destroy(x);
+      return rc;
+    }
+    groups.push_back(sub);
+    tok0.push_back(plan->cu_seqlens[b0]);
+    b0 = b1;
+  }
+  tok0.push_back(T);
+  plan->groups = std::move(groups);
+  plan->group_tok0 = std::move(tok0);
+  return FCP_OK;
+}
+}  // namespace
+
 extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host, const void* v_host,
                                      const void* d_o_host, void* o_host, float* lse_host, void* dq_host, void* dk_host,
                                      void* dv_host, void* workspace, int64_t workspace_bytes, void* stream) {
@@ -563,63 +614,86 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
                   (long long)L.total);
     return FCP_ERR_WORKSPACE;
   }
-  const fcp_params& P = plan->params;
-  const int64_t T = plan->T, D = P.head_dim;
-  char* w = (char*)workspace;
   cudaStream_t st = (cudaStream_t)stream;
-  // Copies that no kernel is waiting for run on two side streams: dO comes in while the forward
-  // pass runs, O and LSE go out while the backward pass runs.  Everything is ordered after the work
-  // already queued on `stream` and is complete when this call returns.
+  if ((rc = build_host_groups(plan, stream)) != FCP_OK) return rc;
+  const fcp_params& P = plan->params;
+  const int64_t D = P.head_dim;
+  const int64_t rq = (int64_t)P.hq * D * 2, rkv = (int64_t)P.hkv * D * 2, rl = (int64_t)P.hq * 4;   // bytes per token
+  char* w = (char*)workspace;
+  const int G = (int)plan->groups.size();
+  // Three streams: inputs of group g+1 come in and results of group g-1 go out while the kernels of
+  // group g run on `stream`.  Everything is ordered after the work already queued on `stream` and is
+  // complete when this call returns.
   struct Side {
     cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t qkv = nullptr, d_o = nullptr, fwd = nullptr, o_out = nullptr;
+    cudaEvent_t start = nullptr, last_out = nullptr;
+    std::vector<cudaEvent_t> up, done;
     ~Side() {
-      if (qkv) cudaEventDestroy(qkv);
-      if (d_o) cudaEventDestroy(d_o);
-      if (fwd) cudaEventDestroy(fwd);
-      if (o_out) cudaEventDestroy(o_out);
+      for (cudaEvent_t e : up) if (e) cudaEventDestroy(e);
+      for (cudaEvent_t e : done) if (e) cudaEventDestroy(e);
+      if (start) cudaEventDestroy(start);
+      if (last_out) cudaEventDestroy(last_out);
       if (in) cudaStreamDestroy(in);
       if (out) cudaStreamDestroy(out);
     }
   } side;
   FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.in, cudaStreamNonBlocking));
   FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.out, cudaStreamNonBlocking));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.qkv, cudaEventDisableTiming));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.d_o, cudaEventDisableTiming));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.fwd, cudaEventDisableTiming));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.o_out, cudaEventDisableTiming));
-
-  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q, q_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k, k_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v, v_host, T * P.hkv * D * 2, cudaMemcpyHostToDevice, st));
-  FCP_CUDA_CHECK(cudaEventRecord(side.qkv, st));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.in, side.qkv, 0));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o, d_o_host, T * P.hq * D * 2, cudaMemcpyHostToDevice, side.in));
-  FCP_CUDA_CHECK(cudaEventRecord(side.d_o, side.in));
-  for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
-    const int hc = std::min(L.heads_per_pass, P.hq - h0);
-    if ((rc = fcp_attn_fwd_merged(plan, w + L.q, w + L.k, w + L.v, h0, hc, (float*)(w + L.o_part), (float*)(w + L.lse_part),
-                                  w + L.o, (float*)(w + L.lse), st)) != FCP_OK)
-      return rc;
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.start, cudaEventDisableTiming));
+  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.last_out, cudaEventDisableTiming));
+  side.up.assign(G, nullptr);
+  side.done.assign(G, nullptr);
+  for (int g = 0; g < G; ++g) {
+    FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.up[g], cudaEventDisableTiming));
+    FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.done[g], cudaEventDisableTiming));
   }
-  FCP_CUDA_CHECK(cudaEventRecord(side.fwd, st));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.fwd, 0));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(o_host, w + L.o, T * P.hq * D * 2, cudaMemcpyDeviceToHost, side.out));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(lse_host, w + L.lse, T * P.hq * 4, cudaMemcpyDeviceToHost, side.out));
-  FCP_CUDA_CHECK(cudaEventRecord(side.o_out, side.out));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.d_o, 0));
-  int64_t scratch = 0;
-  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
-  if ((rc = fcp_attn_bwd(plan, w + L.q, w + L.k, w + L.v, w + L.o, w + L.d_o, (float*)(w + L.lse), w + L.dq, w + L.dk,
-                         w + L.dv, w + L.scratch, scratch, st)) != FCP_OK) {
+  auto drain_sides = [&]() {
     cudaStreamSynchronize(side.in);
     cudaStreamSynchronize(side.out);
-    return rc;
+    cudaStreamSynchronize(st);
+  };
+  FCP_CUDA_CHECK(cudaEventRecord(side.start, st));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.in, side.start, 0));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.start, 0));
+  for (int g = 0; g < G; ++g) {
+    const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q + t0 * rq, (const char*)q_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, side.in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k + t0 * rkv, (const char*)k_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, side.in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v + t0 * rkv, (const char*)v_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, side.in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o + t0 * rq, (const char*)d_o_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, side.in));
+    FCP_CUDA_CHECK(cudaEventRecord(side.up[g], side.in));
   }
-  FCP_CUDA_CHECK(cudaMemcpyAsync(dq_host, w + L.dq, T * P.hq * D * 2, cudaMemcpyDeviceToHost, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(dk_host, w + L.dk, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
-  FCP_CUDA_CHECK(cudaMemcpyAsync(dv_host, w + L.dv, T * P.hkv * D * 2, cudaMemcpyDeviceToHost, st));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.o_out, 0));
+  for (int g = 0; g < G; ++g) {
+    const fcp_plan* sub = plan->groups[g];
+    const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.up[g], 0));
+    for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
+      const int hc = std::min(L.heads_per_pass, P.hq - h0);
+      if ((rc = fcp_attn_fwd_merged(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, h0, hc,
+                                    (float*)(w + L.o_part), (float*)(w + L.lse_part), w + L.o + t0 * rq,
+                                    (float*)(w + L.lse + t0 * rl), st)) != FCP_OK) {
+        drain_sides();
+        return rc;
+      }
+    }
+    int64_t scratch = 0;
+    fcp_plan_workspace_bytes(sub, 1, nullptr, nullptr, &scratch);
+    if ((rc = fcp_attn_bwd(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, w + L.o + t0 * rq,
+                           w + L.d_o + t0 * rq, (float*)(w + L.lse + t0 * rl), w + L.dq + t0 * rq, w + L.dk + t0 * rkv,
+                           w + L.dv + t0 * rkv, w + L.scratch, scratch, st)) != FCP_OK) {
+      drain_sides();
+      return rc;
+    }
+    FCP_CUDA_CHECK(cudaEventRecord(side.done[g], st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.done[g], 0));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, side.out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, side.out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dq_host + t0 * rq, w + L.dq + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, side.out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dk_host + t0 * rkv, w + L.dk + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, side.out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dv_host + t0 * rkv, w + L.dv + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, side.out));
+  }
+  FCP_CUDA_CHECK(cudaEventRecord(side.last_out, side.out));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.last_out, 0));
   FCP_CUDA_CHECK(cudaStreamSynchronize(st));
   return FCP_OK;
 }

@@ -46,6 +46,11 @@ struct fcp_plan {
   int32_t* d_status = nullptr; // [4]: status word, diagnostic
   int sm_count = 0;
 
+  // Sub-plans over runs of consecutive sequences, built and uploaded at the first call of the host
+  // entry point, which pipelines copies and kernels over them (owned by this plan).
+  mutable std::vector<fcp_plan*> groups;
+  mutable std::vector<int64_t> group_tok0;   // first packed token of each group, plus T at the end
+
   // optional kernel timing: ring of event pairs per kernel kind (void* = cudaEvent_t)
   bool profiling = false;
   void* prof_ev[FCP_KERNEL_KINDS][64][2] = {};

@@ -188,10 +188,15 @@ def test_chunked_plan_agrees_with_degree_one_plan():
         assert np.linalg.norm(a[n] - b[n]) <= GRAD_REL * np.linalg.norm(b[n])
 
 
-def test_host_buffer_entry_point_matches_device_path():
+@pytest.mark.parametrize("lens,degs", [
+    ([900, 130], [3, 1]),                                              # one sequence group
+    ([2100, 1800, 2500, 900, 3000, 1500, 2048, 4097, 700, 2600, 1900, 3100],
+     [1, 2, 1, 1, 3, 1, 2, 1, 1, 2, 1, 3]),                           # three groups, pipelined copies and kernels
+])
+def test_host_buffer_entry_point_matches_device_path(lens, degs):
     from paper_2602_21788_b200 import fcp
     from paper_2602_21788_b200.runner import run_fwd_bwd
-    w = _wl([900, 130], [3, 1], 4, 2, 128, seed=7)
+    w = _wl(lens, degs, 4, 2, 128, seed=7)
     q, k, v, do = w.tensors()
     ref = run_fwd_bwd(w, q, k, v, do)
     plan = ref["state"].plan
@@ -211,6 +216,12 @@ def test_host_buffer_entry_point_matches_device_path():
     assert np.array_equal(back(ho), ref["o"]) and np.array_equal(hlse.numpy(), ref["lse"])
     assert np.array_equal(back(hdk), ref["dk"]) and np.array_equal(back(hdv), ref["dv"])
     assert np.linalg.norm(back(hdq) - ref["dq"]) <= 1e-2 * np.linalg.norm(ref["dq"])
+    assert plan.device_status()[0] == 0
+    # a second call reuses the sequence groups built by the first
+    ho.zero_(); hdk.zero_()
+    fcp.fcp_attn_fwd_bwd_host(plan, hq_, hk_, hv_, hdo_, ho, hlse, hdq, hdk, hdv, ws, nbytes,
+                              torch.cuda.current_stream().cuda_stream)
+    assert np.array_equal(back(ho), ref["o"]) and np.array_equal(back(hdk), ref["dk"])
     with pytest.raises(fcp.FcpError) as e:
         fcp.fcp_attn_fwd_bwd_host(plan, hq_, hk_, hv_, hdo_, ho, hlse, hdq, hdk, hdv, ws, 1024, 0)
     assert e.value.status == fcp.FCP_ERR_WORKSPACE
