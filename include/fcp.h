@@ -18,6 +18,12 @@
  *     objects (host tables plus, after fcp_plan_upload, a device copy of them).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Compute calls only
  *     enqueue work on it; they do not synchronise and do not allocate device memory.
+ *   - Calls that use one plan must be stream-ordered with respect to each other: the plan's device
+ *     copy holds the status words and the work counter of the backward grid, so two compute calls
+ *     on the same plan that overlap on the GPU (different streams, different threads) race.  Use
+ *     one plan per concurrent stream.
+ *   - The device status words are sticky: once a kernel has recorded FCP_ERR_TIMEOUT they keep it
+ *     for the life of the plan's device copy (fcp_last_device_status reports the first failure).
  *   - Tensors are packed token-major ("THD"), row-major, bf16:
  *         q, o, d_o, dq : [T][hq][D]        k, v, dk, dv : [T][hkv][D]
  *     T = total tokens of the batch, D = head_dim in {64, 128}, hq % hkv == 0; query head h reads
@@ -105,20 +111,24 @@ int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B
 #define FCP_TABLE_BWD_UNITS     8  /* [n_bwd_units][8]          derived                               */
 #define FCP_TABLE_BWD_QRANGES   9  /* [n_bwd_qranges][4]        derived                               */
 #define FCP_TABLE_MERGE_UNITS  10  /* [n_merge_units][4]        derived                               */
-#define FCP_TABLE_BWD_WORK     11  /* [n_bwd_units*hkv][2]      derived: (unit, kv head) in execution order */
+#define FCP_TABLE_BWD_WORK     11  /* [n_bwd_units]             derived: backward units in execution order (per KV head) */
+#define FCP_TABLE_FUSED_UNITS  12  /* [n_fused_units][16]       derived: work units of fcp_attn_fwd_fused       */
 
 /* fcp_plan_get: *host_ptr = first element of the table, *count = number of int32 elements. */
 int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count);
 
 /* Scalar facts about a plan: which in {0: T, 1: R (partial rows), 2: n_pairs, 3: n_items,
  * 4: n_fwd_units, 5: n_bwd_units, 6: n_merge_units, 7: B, 8: the leading merge units that belong
- * to Q chunks with two or more slots (all that fcp_attn_fwd_merged has to merge)}.                */
+ * to Q chunks with two or more slots (all that fcp_attn_fwd_merged has to merge), 9: n_fused_units}. */
 int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value);
 
 /* Bytes the caller must provide: o_partial = R*heads_per_pass*D*4, lse_partial = R*heads_per_pass*4,
  * bwd_scratch (all hq heads at once) for fcp_attn_bwd.  Any output pointer may be NULL.          */
 int fcp_plan_workspace_bytes(const fcp_plan* plan, int32_t heads_per_pass, int64_t* o_partial_bytes,
                              int64_t* lse_partial_bytes, int64_t* bwd_scratch_bytes);
+/* Scratch bytes of fcp_attn_bwd_heads for a pass over kv_head_count KV heads (and their query
+ * heads): about 4*T*(kv_head_count*hq/hkv)*D bytes.                                               */
+int fcp_plan_bwd_scratch_bytes(const fcp_plan* plan, int32_t kv_head_count, int64_t* bytes);
 
 /* Copies the plan's work tables to the current device (the only device allocation the library
  * makes; freed by fcp_plan_destroy).  Must precede the compute calls.  Synchronous.              */
@@ -153,6 +163,22 @@ int fcp_attn_fwd_merged(const fcp_plan* plan, const void* q, const void* k, cons
                         void* o, float* lse, void* stream);
 
 /* ------------------------------------------------------------------------------------------
+ * fcp_attn_fwd_fused — device.  The forward pass with the merge done on the fly: all items of a Q
+ * chunk are scheduled onto one CTA, which sweeps the KV ranges of every block pair of the chunk
+ * (the same pairs fcp_attn_fwd executes, FCP_TABLE_FUSED_UNITS lists them per work unit) in a
+ * single online softmax and writes o [T][hq][D] bf16 and lse [T][hq] fp32 directly (Eq. 1; the
+ * merge of Sec. 3.2's ring steps is the re-association the online softmax performs anyway).  No
+ * partial buffer is needed.  Adjacent Q chunks of a causal plan are tiled as one run of rows, so
+ * no tile is cut at a chunk edge and the running time does not depend on the degrees.  Results
+ * agree with fcp_attn_fwd + fcp_lse_merge to rounding (the summation order differs).
+ * o_f32 is optional (NULL to skip): the same output [T][hq][D] before the rounding to bf16.
+ * Heads [head_begin, head_begin+head_count).  Asynchronous on `stream`.
+ */
+int fcp_attn_fwd_fused(const fcp_plan* plan, const void* q, const void* k, const void* v,
+                       int32_t head_begin, int32_t head_count, void* o, float* o_f32, float* lse,
+                       void* stream);
+
+/* ------------------------------------------------------------------------------------------
  * fcp_lse_merge — device.  Exact combination of the slots of every (token, head):
  *     LSE = m + log sum_s exp(lse_s - m),  o = sum_s exp(lse_s - LSE) * o_s     (m = max_s lse_s)
  * (the re-association of the softmax sum implied by ring-style CP, Sec. 3.2).
@@ -177,17 +203,31 @@ int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void*
                  const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* scratch,
                  int64_t scratch_bytes, void* stream);
 
+/* fcp_attn_bwd_heads — device.  fcp_attn_bwd restricted to the KV heads [kv_head_begin,
+ * kv_head_begin + kv_head_count) and the hq/hkv query heads of each: writes dk, dv of those KV
+ * heads and dq of those query heads, leaves the other heads of the outputs untouched.  KV heads are
+ * independent problems (no sum crosses them), so passes over disjoint ranges give the result of
+ * one call over all heads; this bounds the scratch (fcp_plan_bwd_scratch_bytes) and is the unit by
+ * which the backward pass can be split over GPUs.  All tensors keep their full [T][heads][D] shape.
+ */
+int fcp_attn_bwd_heads(const fcp_plan* plan, const void* q, const void* k, const void* v,
+                       const void* o, const void* d_o, const float* lse, int32_t kv_head_begin,
+                       int32_t kv_head_count, void* dq, void* dk, void* dv, void* scratch,
+                       int64_t scratch_bytes, void* stream);
+
 /* ------------------------------------------------------------------------------------------
  * fcp_attn_fwd_bwd_host — the whole path from HOST buffers: copies q, k, v, d_o to the device,
- * runs fcp_attn_fwd_merged (in head passes that fit the workspace) and fcp_attn_bwd, and copies
- * o, lse, dq, dk, dv back.  `workspace` is a caller-owned DEVICE buffer of `workspace_bytes` >=
- * fcp_host_workspace_bytes(plan); host pointers should be pinned for the copies to be asynchronous.
+ * runs fcp_attn_fwd_fused and fcp_attn_bwd, and copies o, lse, dq, dk, dv back.  `workspace` is a
+ * caller-owned DEVICE buffer of `workspace_bytes` >= fcp_host_workspace_bytes(plan); host pointers
+ * should be pinned for the copies to be asynchronous.
  * The batch is cut into up to 8 runs of consecutive sequences (packed tensors are token-major, so a
  * run is one contiguous slice of every tensor); the inputs of the next run come in and the results
  * of the previous one go out while the kernels of the current run execute (two internal copy
- * streams, ordered after the work already queued on `stream`).  The first call on a plan builds and
- * uploads the plans of the runs (small device allocations, freed by fcp_plan_destroy).
- * Synchronises `stream` before returning; every output is complete then.
+ * streams, ordered after the work already queued on `stream`).  The first call on a plan is the
+ * one exception to "compute calls do not allocate": it builds and uploads the plans of the runs
+ * and creates the copy streams and events (small allocations, all released by fcp_plan_destroy).
+ * Synchronises `stream` before returning; every output is complete then.  On an error return the
+ * work already queued has been waited for, so nothing writes into the caller's buffers afterwards.
  */
 int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes);
 int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host,
@@ -195,8 +235,9 @@ int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* 
                           void* dq_host, void* dk_host, void* dv_host, void* workspace,
                           int64_t workspace_bytes, void* stream);
 
-/* Device-side status word of the last kernels run with this plan (0 = fine; FCP_ERR_TIMEOUT if a
- * bounded wait inside a kernel expired).  Synchronises the device.                               */
+/* Device-side status words of the kernels run with this plan so far: status[0] = 0 while all is
+ * fine, FCP_ERR_TIMEOUT once a bounded wait inside a kernel has expired (sticky, first failure
+ * wins); status[1] = code of the wait that gave up, status[2] = its CTA.  Synchronises the device. */
 int fcp_last_device_status(const fcp_plan* plan, int32_t* status);
 
 /* ------------------------------------------------------------------------------------------
@@ -224,8 +265,9 @@ int fcp_last_device_status(const fcp_plan* plan, int32_t* status);
  *   - All calls on a device share the one array and it keeps the previous call's contents (the
  *     function clears what has to start from zero).  Two calls that can overlap on the GPU, on
  *     different streams or from different threads, corrupt each other: serialise them.
- *   - The plan's host tables are read by the asynchronous copies: keep the plan alive until the
- *     stream has passed this call.
+ *   - The plan's host tables are read by the asynchronous copies at the moment those copies execute,
+ *     not when this function returns: keep the plan alive and unchanged for as long as any copy
+ *     issued by this call can still run.
  * fcp_noalloc_device_status reads the status words of the last such call on the current device
  * (synchronises the device; 0 = fine, FCP_ERR_TIMEOUT if a bounded wait in the kernel expired).
  */

@@ -3,7 +3,7 @@
 Eq. 4 models the compute time of one rank of a CP group as  sum_k (alpha1 (1 + eta_k) L_k^2 + alpha2 L_k)
 / d + beta1.  Here all d virtual ranks of a sequence run in one grid on one GPU, so what can be timed
 is the sum over the ranks:  T(L, d) = alpha1 L^2 + alpha2 L + beta1 d  (causal attention: eta = 0).
-`measure_grid` times the whole hot path (forward over the plan, merge, backward) through the C ABI on
+`measure_grid` times the whole hot path (forward over the plan with the merge on the fly, backward) through the C ABI on
 batches of equal-length sequences that fill the GPU; `fit` solves the least-squares problem for
 (alpha1, alpha2, beta1); `relative_errors` gives the estimation error the paper reports in its
 cost-model table (predicted against measured time of mixed batches).  The fitted coefficients are
@@ -16,6 +16,9 @@ from __future__ import annotations
 import argparse
 
 import numpy as np
+
+# Last fit on a B200 (32 query / 8 KV heads, head_dim 128), ms units; see `main` for how it is taken.
+B200_COEFFS = dict(alpha1=3.304068e-08, alpha2=1.535782e-06, beta1=1.788982e-02)
 
 
 def design_row(seqlens, cp_degrees):
@@ -49,7 +52,7 @@ def relative_errors(coeffs, batches, times_ms):
 # measurement (GPU)
 # ------------------------------------------------------------------------------------------------
 def time_batch(seqlens, cp_degrees, hq, hkv, head_dim, reps=5, warmup=2, seed=0) -> float:
-    """Median ms of forward + merge + backward for one synthetic batch (inputs resident on the GPU)."""
+    """Median ms of fused forward + backward for one synthetic batch (inputs resident on the GPU)."""
     import torch
 
     from . import synth
@@ -61,19 +64,19 @@ def time_batch(seqlens, cp_degrees, hq, hkv, head_dim, reps=5, warmup=2, seed=0)
     g = torch.Generator(device="cuda")
     g.manual_seed(seed)
 
-    def bits(h):   # N(0,1) rounded to bf16, as in the workloads (values do not change the timing)
-        return torch.randn((T, h, head_dim), device="cuda", generator=g).bfloat16().view(torch.int16).cpu().numpy().view(np.uint16)
+    def draw(h):   # N(0,1) rounded to bf16, as in the workloads (values do not change the timing)
+        return torch.randn((T, h, head_dim), device="cuda", generator=g, dtype=torch.bfloat16)
 
-    ds = DeviceState(w, bits(hq), bits(hkv), bits(hkv), bits(hq))
+    ds = DeviceState(w, draw(hq), draw(hkv), draw(hkv), draw(hq), partials=False)
     for _ in range(warmup):
-        ds.forward()
+        ds.forward_fused()
         ds.backward()
     torch.cuda.synchronize()
     out = []
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        ds.forward()
+        ds.forward_fused()
         ds.backward()
         e1.record()
         torch.cuda.synchronize()
@@ -119,7 +122,7 @@ def main():
                                  coeffs=dict(alpha1=c["alpha1"], alpha2=c["alpha2"], alpha3=0.0, beta1=c["beta1"], beta2=0.0, v=1.0))
     lines = ["# Cost-model coefficients of Eq. 4 fitted on one B200 (`python -m paper_2602_21788_b200.costfit`)", "",
              f"Shape: {hq} query / {hkv} KV heads, head_dim {D}, causal, bf16; batches of 65536 tokens of equal-length sequences;",
-             "time = forward over the plan + merge + backward (median of 5, CUDA events).", "",
+             "time = forward over the plan with the merge on the fly + backward (median of 5, CUDA events).", "",
              f"alpha1 = {c['alpha1']:.6e} ms/token^2, alpha2 = {c['alpha2']:.6e} ms/token, beta1 = {c['beta1']:.6e} ms per virtual rank", "",
              f"Fit residual over the {len(times)} grid points: mean {100 * grid_err.mean():.2f} %, max {100 * grid_err.max():.2f} %.",
              "Estimation error on held-out mixed batches (`llama8b_64k` recipe, seeds 0-4): "

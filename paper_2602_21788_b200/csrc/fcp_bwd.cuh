@@ -20,8 +20,9 @@
 // as C1 has read S^T, and T2 of the next tile as soon as C3 has drained dQ, so the tensor core, the
 // math warps and the drain warps work on different tiles at the same time.
 //
-// Work items are handed out through a global counter in plan order (one (sequence, KV head) panel
-// after the other, keys ascending), so that the dQ rows being reduced into stay in L2.
+// Work items are handed out through a global counter: KV heads one after the other, within a head
+// the units in plan order (one sequence after the other, keys ascending), so that the dQ rows being
+// reduced into stay in L2.
 #pragma once
 #include "fcp_plan.hpp"
 #include "sm100_ptx.cuh"
@@ -55,14 +56,16 @@ struct BwdSmem {
 struct BwdArgs {
   const int32_t* units;     // [n_units][8]
   const int32_t* qranges;   // [n][4]
-  const int32_t* work;      // [n_work][2]: (unit, kv head) in execution order
-  int32_t n_work, hq, hkv;
+  const int32_t* work;      // [n_units]: units in execution order; work item w = (work[w % n_units], hk_begin + w / n_units)
+  int32_t n_work, n_units, hq, hkv;
+  int32_t hk_begin;         // first KV head of this pass
+  int32_t hq_acc;           // query heads held by dq_acc / delta_t / lse2_t: those of the pass, numbered from 0
   int32_t* counter;         // work counter, zero before the launch
   int64_t T, t_stride;
   float scale, scale_log2;
-  const float* delta_t;     // [hq][t_stride], already multiplied by the softmax scale
-  const float* lse2_t;      // [hq][t_stride], log2 units
-  float* dq_acc;            // [T][hq][D] fp32, zero-initialised
+  const float* delta_t;     // [hq_acc][t_stride], already multiplied by the softmax scale
+  const float* lse2_t;      // [hq_acc][t_stride], log2 units
+  float* dq_acc;            // [T][hq_acc][D] fp32, zero-initialised
   __nv_bfloat16* dk;        // [T][hkv][D]
   __nv_bfloat16* dv;
   int32_t* status;
@@ -221,8 +224,8 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         ok = mbar_wait(BAR(B_WEMPTY + slot), ((n >> 1) & 1) ^ 1, wctx, 112);
         if (!ok) break;
         const bool last = w >= a.n_work;
-        const int unit = last ? -1 : __ldg(a.work + 2 * w);
-        const int hk = last ? 0 : __ldg(a.work + 2 * w + 1);
+        const int unit = last ? -1 : __ldg(a.work + w % a.n_units);
+        const int hk = last ? 0 : a.hk_begin + w / a.n_units;
         work_ring[2 * slot] = unit;
         work_ring[2 * slot + 1] = hk;
         mbar_arrive(BAR(B_WFULL + slot));     // release: the two stores above are visible to the waiters
@@ -344,7 +347,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const float* my_rows = (mtid < 128 ? a.lse2_t : a.delta_t) + (mtid & 127);
     auto load_row = [&](const BwdIter& x, int hk) -> float {
       const int64_t t = (int64_t)x.q_row + (mtid & 127);
-      return t < a.T ? __ldg(my_rows + (int64_t)(hk * g + x.hh) * a.t_stride + x.q_row) : 0.f;
+      return t < a.T ? __ldg(my_rows + (int64_t)((hk - a.hk_begin) * g + x.hh) * a.t_stride + x.q_row) : 0.f;
     };
     uint32_t n = 0, it = 0;
     bool ok = true;
@@ -480,15 +483,15 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       BwdIter iter;
 #pragma unroll 1
       for (iter.init(U, a.qranges, g); iter.valid; iter.advance(), ++it) {
-        const int h = hk * g + iter.hh;
+        const int h = (hk - a.hk_begin) * g + iter.hh;   // head index within the accumulators of this pass
         const int q_row = iter.q_row, q_valid = iter.q_valid;
         ok = mbar_wait_warp(BAR(B_DQFULL), it & 1, wctx, 132);
         if (!ok) break;
         tc_fence_after();
         if constexpr (DQ_T) {
           // thread = head-dim index, columns = queries: a warp adds 32 consecutive floats per query.
-          char* dst = reinterpret_cast<char*>(a.dq_acc + ((int64_t)q_row * a.hq + h) * D + row);
-          const int64_t stride = (int64_t)a.hq * D * 4;
+          char* dst = reinterpret_cast<char*>(a.dq_acc + ((int64_t)q_row * a.hq_acc + h) * D + row);
+          const int64_t stride = (int64_t)a.hq_acc * D * 4;
           if (q_valid == 128) {
             // whole tile into registers, columns handed back at once, then the reductions: they are
             // slow (L2 round trips) and must not sit between the tile and the issuer's next product
@@ -540,7 +543,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
           }
         } else {
-          float* dst = a.dq_acc + (((int64_t)q_row + row) * a.hq + h) * D;
+          float* dst = a.dq_acc + (((int64_t)q_row + row) * a.hq_acc + h) * D;
 #pragma unroll 1
           for (int c16 = 0; c16 < D / 16; ++c16) {
             uint32_t qv[16];

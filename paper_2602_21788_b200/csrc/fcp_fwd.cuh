@@ -52,6 +52,7 @@ struct FwdArgs {
   float* lse_partial;     // [R][head_count]
   __nv_bfloat16* o_direct;   // [T][hq][D] or nullptr: final output of Q chunks that have a single slot
   float* lse_direct;         // [T][hq]
+  float* o_f32_direct;       // [T][hq][D] or nullptr: the rows written to o_direct before their rounding to bf16
   int32_t* status;        // [4]
 };
 
@@ -407,6 +408,22 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             }
           }
           if (row < rows_s) a.lse_direct[orow] = lse_row;
+          if (a.o_f32_direct != nullptr) {
+            float* fp = a.o_f32_direct + orow * D;
+#pragma unroll 1
+            for (int c = 0; c < D / 32; ++c) {
+              uint32_t ov[32];
+              tmem_ld32(t_o + c * 32, ov);
+              tc_wait_ld();
+              if (row < rows_s) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                  *reinterpret_cast<float4*>(fp + c * 32 + i) =
+                      make_float4(__uint_as_float(ov[i]) * inv_l, __uint_as_float(ov[i + 1]) * inv_l,
+                                  __uint_as_float(ov[i + 2]) * inv_l, __uint_as_float(ov[i + 3]) * inv_l);
+              }
+            }
+          }
         } else {
           const int64_t prow = prow0 + s * 128 + row;
           float* op = a.o_partial + (prow * a.head_count + hl) * D;

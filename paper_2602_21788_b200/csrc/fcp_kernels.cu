@@ -72,7 +72,7 @@ struct ProfScope {
   cudaStream_t st;
   int slot = -1;
   ProfScope(const fcp_plan* p, int k, cudaStream_t s) : plan(p), kind(k), st(s) {
-    if (plan->profiling && plan->prof_ev[kind][0][0]) {
+    if (plan && plan->profiling && plan->prof_ev[kind][0][0]) {
       slot = (int)(plan->prof_n[kind] % 64);
       cudaEventRecord((cudaEvent_t)plan->prof_ev[kind][slot][0], st);
     }
@@ -153,15 +153,20 @@ __global__ void __launch_bounds__(256) fcp_merge_kernel(const int32_t* __restric
 // ---------------------------------------------------------------------------------------------
 template <int D>
 __global__ void __launch_bounds__(256) fcp_delta_kernel(const __nv_bfloat16* __restrict__ o, const __nv_bfloat16* __restrict__ d_o,
-                                                        const float* __restrict__ lse, int64_t T, int hq, int64_t t_stride, float scale,
-                                                        float* __restrict__ delta_t, float* __restrict__ lse2_t) {
+                                                        const float* __restrict__ lse, int64_t T, int hq, int h0, int hc,
+                                                        int64_t t_stride, float scale, float* __restrict__ delta_t,
+                                                        float* __restrict__ lse2_t) {
+  // heads [h0, h0 + hc) of the [T][hq][D] tensors; the outputs hold hc heads, numbered from 0
   constexpr int TPR = D / 8;
-  const int64_t row = ((int64_t)blockIdx.x * 256 + threadIdx.x) / TPR;   // (token, head) row
+  const int64_t row = ((int64_t)blockIdx.x * 256 + threadIdx.x) / TPR;   // (token, head of the pass) row
   const int sub = threadIdx.x % TPR;
+  const int64_t t = row / hc;
+  const int hl = (int)(row - t * hc);
+  const int64_t src = t * hq + h0 + hl;
   float acc = 0.f;
-  if (row < T * hq) {
-    const uint4 a = *reinterpret_cast<const uint4*>(o + row * D + sub * 8);
-    const uint4 b = *reinterpret_cast<const uint4*>(d_o + row * D + sub * 8);
+  if (row < T * hc) {
+    const uint4 a = *reinterpret_cast<const uint4*>(o + src * D + sub * 8);
+    const uint4 b = *reinterpret_cast<const uint4*>(d_o + src * D + sub * 8);
     const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
     const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
 #pragma unroll
@@ -172,24 +177,28 @@ __global__ void __launch_bounds__(256) fcp_delta_kernel(const __nv_bfloat16* __r
   }
 #pragma unroll
   for (int off = TPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-  if (row < T * hq && sub == 0) {
-    const int64_t t = row / hq;
-    const int h = (int)(row % hq);
-    delta_t[h * t_stride + t] = acc * scale;
-    lse2_t[h * t_stride + t] = lse[row] * 1.4426950408889634f;
+  if (row < T * hc && sub == 0) {
+    delta_t[hl * t_stride + t] = acc * scale;
+    lse2_t[hl * t_stride + t] = lse[src] * 1.4426950408889634f;
   }
 }
 
-// fp32 dQ accumulator -> bf16
+// fp32 dQ accumulator [T][hc][D] -> bf16 dq [T][hq][D], heads [h0, h0 + hc); n8 = T*hc*D/8 groups of
+// eight values, row8 = hc*D/8 groups per token of the accumulator
 __global__ void __launch_bounds__(256) fcp_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq,
-                                                             int64_t n8) {
+                                                             int64_t n8, int64_t row8, int64_t dst_row8, int64_t dst_off8) {
   for (int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x; i < n8; i += (int64_t)gridDim.x * 256) {
     const float4 a = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i);
     const float4 b = __ldcs(reinterpret_cast<const float4*>(acc) + 2 * i + 1);
     uint4 pk;
     pk.x = pack_bf16(a.x, a.y); pk.y = pack_bf16(a.z, a.w);
     pk.z = pack_bf16(b.x, b.y); pk.w = pack_bf16(b.z, b.w);
-    reinterpret_cast<uint4*>(dq)[i] = pk;
+    int64_t j = i;
+    if (row8 != dst_row8) {
+      const int64_t t = i / row8;
+      j = t * dst_row8 + dst_off8 + (i - t * row8);
+    }
+    reinterpret_cast<uint4*>(dq)[j] = pk;
   }
 }
 
@@ -209,20 +218,21 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   }
   plan->device = dev;
   plan->sm_count = prop.multiProcessorCount;
-  const std::vector<int32_t>* tabs[7] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges,
-                                         &plan->merge_units, &plan->slot_offset, &plan->slot_rows, &plan->bwd_work};
-  size_t off[8];
+  constexpr int NT = 8;
+  const std::vector<int32_t>* tabs[NT] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges, &plan->merge_units,
+                                          &plan->slot_offset, &plan->slot_rows, &plan->bwd_work, &plan->fused_units};
+  size_t off[NT + 1];
   size_t total = 256;  // status words first
-  for (int i = 0; i < 7; ++i) {
+  for (int i = 0; i < NT; ++i) {
     off[i] = total;
     total += (tabs[i]->size() * 4 + 255) / 256 * 256;
   }
-  off[7] = total;
+  off[NT] = total;
   void* blob = nullptr;
   FCP_CUDA_CHECK(cudaMalloc(&blob, total));
   cudaStream_t st = (cudaStream_t)stream;
   cudaError_t e = cudaMemsetAsync(blob, 0, 256, st);
-  for (int i = 0; i < 7 && e == cudaSuccess; ++i)
+  for (int i = 0; i < NT && e == cudaSuccess; ++i)
     if (!tabs[i]->empty())
       e = cudaMemcpyAsync((char*)blob + off[i], tabs[i]->data(), tabs[i]->size() * 4, cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
@@ -240,6 +250,7 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   plan->d_slot_offset = (int32_t*)((char*)blob + off[4]);
   plan->d_slot_rows = (int32_t*)((char*)blob + off[5]);
   plan->d_bwd_work = (int32_t*)((char*)blob + off[6]);
+  plan->d_fused_units = (int32_t*)((char*)blob + off[7]);
   // opt in to the large dynamic shared memory of the tensor-core kernels once
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::DYN_BYTES));
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::DYN_BYTES));
@@ -286,6 +297,11 @@ extern "C" int fcp_plan_destroy(fcp_plan* plan) {
   if (!plan) return FCP_OK;
   for (fcp_plan* g : plan->groups) fcp_plan_destroy(g);
   plan->groups.clear();
+  for (void* e : plan->host_events) if (e) cudaEventDestroy((cudaEvent_t)e);
+  plan->host_events.clear();
+  if (plan->host_in) cudaStreamDestroy((cudaStream_t)plan->host_in);
+  if (plan->host_out) cudaStreamDestroy((cudaStream_t)plan->host_out);
+  plan->host_in = plan->host_out = nullptr;
   fcp_plan_set_profiling(plan, 0);
   if (plan->d_blob) cudaFree(plan->d_blob);
   delete plan;
@@ -335,12 +351,14 @@ static int check_heads(const fcp_plan* plan, int head_begin, int head_count) {
 }
 
 namespace {
+// `fused`: run the merge-on-the-fly units (every row goes straight to o_direct / lse_direct, no partials)
 int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin, int32_t head_count,
-               float* o_partial, float* lse_partial, void* o_direct, float* lse_direct, void* stream) {
+               float* o_partial, float* lse_partial, void* o_direct, float* lse_direct, float* o_f32_direct, bool fused,
+               void* stream) {
   int rc = check_plan(plan);
   if (rc != FCP_OK) return rc;
-  if (!q || !k || !v || !o_partial || !lse_partial) {
-    fcp_set_error("fcp_attn_fwd: NULL buffer");
+  if (!q || !k || !v || (!fused && (!o_partial || !lse_partial)) || (fused && (!o_direct || !lse_direct))) {
+    fcp_set_error("forward attention: NULL buffer");
     return FCP_ERR_INVALID_ARG;
   }
   if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
@@ -350,8 +368,8 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
   if ((rc = make_thd_map(&tk, k, plan->T, P.hkv, P.head_dim, 128)) != FCP_OK) return rc;
   if ((rc = make_thd_map(&tv, v, plan->T, P.hkv, P.head_dim, 128)) != FCP_OK) return rc;
   FwdArgs a;
-  a.units = plan->d_fwd_units;
-  a.n_units = (int32_t)(plan->fwd_units.size() / FCP_FWD_UNIT_W);
+  a.units = fused ? plan->d_fused_units : plan->d_fwd_units;
+  a.n_units = (int32_t)((fused ? plan->fused_units.size() : plan->fwd_units.size()) / FCP_FWD_UNIT_W);
   a.head_begin = head_begin;
   a.head_count = head_count;
   a.hq = P.hq;
@@ -361,6 +379,7 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
   a.lse_partial = lse_partial;
   a.o_direct = (__nv_bfloat16*)o_direct;
   a.lse_direct = lse_direct;
+  a.o_f32_direct = o_f32_direct;
   a.status = plan->d_status;
   const int64_t n_work = (int64_t)a.n_units * head_count;
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
@@ -394,7 +413,12 @@ int launch_merge(const fcp_plan* plan, const float* o_partial, const float* lse_
 
 extern "C" int fcp_attn_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
                             int32_t head_count, float* o_partial, float* lse_partial, void* stream) {
-  return launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, nullptr, nullptr, stream);
+  return launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, nullptr, nullptr, nullptr, false, stream);
+}
+
+extern "C" int fcp_attn_fwd_fused(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
+                                  int32_t head_count, void* o, float* o_f32, float* lse, void* stream) {
+  return launch_fwd(plan, q, k, v, head_begin, head_count, nullptr, nullptr, o, lse, o_f32, true, stream);
 }
 
 extern "C" int fcp_attn_fwd_merged(const fcp_plan* plan, const void* q, const void* k, const void* v, int32_t head_begin,
@@ -404,7 +428,7 @@ extern "C" int fcp_attn_fwd_merged(const fcp_plan* plan, const void* q, const vo
     fcp_set_error("fcp_attn_fwd_merged: NULL output");
     return FCP_ERR_INVALID_ARG;
   }
-  int rc = launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, o, lse, stream);
+  int rc = launch_fwd(plan, q, k, v, head_begin, head_count, o_partial, lse_partial, o, lse, nullptr, false, stream);
   if (rc != FCP_OK) return rc;
   return launch_merge(plan, o_partial, lse_partial, head_begin, head_count, o, nullptr, lse, plan->n_merge_multi, stream);
 }
@@ -423,41 +447,49 @@ extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const
                       (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W), stream);
 }
 
-extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
-                            const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* scratch,
-                            int64_t scratch_bytes, void* stream) {
-  int rc = check_plan(plan);
-  if (rc != FCP_OK) return rc;
-  if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv || !scratch) {
-    fcp_set_error("fcp_attn_bwd: NULL buffer");
-    return FCP_ERR_INVALID_ARG;
-  }
+namespace {
+// Everything the backward launches need besides the caller's tensors: device tables, status words,
+// work counter, SM count.  fcp_attn_bwd_heads takes them from the uploaded plan, fcp_attn_bwd_noalloc
+// from the built-in arena.
+struct BwdTables {
+  const int32_t *units, *qranges, *order;
+  int32_t* status;
+  int32_t* counter;
+  int sm_count;
+};
+
+// scratch layout: [dq fp32 accumulator T*hc*D] [delta_t hc*Tpad] [lse2_t hc*Tpad], hc = query heads of the pass
+int64_t bwd_scratch_need(const fcp_plan* plan, int kv_heads) {
+  const int64_t hc = (int64_t)kv_heads * (plan->params.hq / plan->params.hkv);
+  return plan->T * hc * plan->params.head_dim * 4 + 2 * bwd_tpad(plan->T) * hc * 4;
+}
+
+// Launches of one backward pass over KV heads [hk0, hk0 + hkc): clear, delta, main kernel, dQ conversion.
+// `prof` may be NULL (no event timing).
+int run_bwd(const fcp_plan* plan, const BwdTables& tb, const void* q, const void* k, const void* v, const void* o,
+            const void* d_o, const float* lse, int hk0, int hkc, void* dq, void* dk, void* dv, void* scratch,
+            const fcp_plan* prof, cudaStream_t st) {
   const fcp_params& P = plan->params;
   const int64_t T = plan->T, D = P.head_dim;
-  int64_t need = 0;
-  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &need);
-  if (scratch_bytes < need) {
-    fcp_set_error("fcp_attn_bwd: scratch of %lld bytes, %lld needed", (long long)scratch_bytes, (long long)need);
-    return FCP_ERR_WORKSPACE;
-  }
-  cudaStream_t st = (cudaStream_t)stream;
+  const int g = P.hq / P.hkv;
+  const int h0 = hk0 * g, hc = hkc * g;
+  const int64_t need = bwd_scratch_need(plan, hkc);
   const int64_t tpad = bwd_tpad(T);
   float* dq_acc = (float*)scratch;
-  float* delta_t = dq_acc + T * P.hq * D;
-  float* lse2_t = delta_t + tpad * P.hq;
+  float* delta_t = dq_acc + T * hc * D;
+  float* lse2_t = delta_t + tpad * hc;
+  int rc;
   {
-    ProfScope prof(plan, 2, st);
+    ProfScope ps(prof, 2, st);
     FCP_CUDA_CHECK(cudaMemsetAsync(scratch, 0, (size_t)need, st));
-    FCP_CUDA_CHECK(cudaMemsetAsync(plan->d_status + 16, 0, sizeof(int32_t), st));   // work counter of the backward grid
-    const int64_t rows = T * P.hq;
-    const int tpr = (int)D / 8;
-    const int64_t blocks = (rows * tpr + 255) / 256;
+    FCP_CUDA_CHECK(cudaMemsetAsync(tb.counter, 0, sizeof(int32_t), st));
+    const int64_t blocks = (T * hc * (D / 8) + 255) / 256;
     if (D == 128)
       fcp_delta_kernel<128><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                              tpad, P.scale, delta_t, lse2_t);
+                                                              h0, hc, tpad, P.scale, delta_t, lse2_t);
     else
       fcp_delta_kernel<64><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                             tpad, P.scale, delta_t, lse2_t);
+                                                             h0, hc, tpad, P.scale, delta_t, lse2_t);
     FCP_CUDA_CHECK(cudaGetLastError());
   }
   CUtensorMap tq, tk, tv, tdo;
@@ -466,13 +498,16 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   if ((rc = make_thd_map(&tv, v, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
   if ((rc = make_thd_map(&tdo, d_o, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
   BwdArgs a;
-  a.units = plan->d_bwd_units;
-  a.qranges = plan->d_bwd_qranges;
-  a.work = plan->d_bwd_work;
-  a.n_work = (int32_t)(plan->bwd_work.size() / 2);
-  a.counter = plan->d_status + 16;
+  a.units = tb.units;
+  a.qranges = tb.qranges;
+  a.work = tb.order;
+  a.n_units = (int32_t)plan->bwd_work.size();
+  a.n_work = a.n_units * hkc;
+  a.counter = tb.counter;
   a.hq = P.hq;
   a.hkv = P.hkv;
+  a.hk_begin = hk0;
+  a.hq_acc = hc;
   a.T = T;
   a.t_stride = tpad;
   a.scale = P.scale;
@@ -482,10 +517,10 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
   a.dq_acc = dq_acc;
   a.dk = (__nv_bfloat16*)dk;
   a.dv = (__nv_bfloat16*)dv;
-  a.status = plan->d_status;
-  const int grid = (int)std::min<int64_t>(a.n_work, plan->sm_count);
+  a.status = tb.status;
+  const int grid = (int)std::min<int64_t>(a.n_work, tb.sm_count);
   if (grid > 0) {
-    ProfScope prof(plan, 3, st);
+    ProfScope ps(prof, 3, st);
     if (D == 128)
       fcp_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
     else
@@ -493,13 +528,57 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
     FCP_CUDA_CHECK(cudaGetLastError());
   }
   {
-    const int64_t n8 = T * P.hq * D / 8;
-    const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)plan->sm_count * 16);
-    ProfScope prof(plan, 4, st);
-    fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8);
+    const int64_t n8 = T * hc * D / 8;
+    const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)tb.sm_count * 16);
+    ProfScope ps(prof, 4, st);
+    fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8, hc * D / 8, P.hq * D / 8, h0 * D / 8);
     FCP_CUDA_CHECK(cudaGetLastError());
   }
   return FCP_OK;
+}
+}  // namespace
+
+extern "C" int fcp_plan_bwd_scratch_bytes(const fcp_plan* plan, int32_t kv_head_count, int64_t* bytes) {
+  if (!plan || !bytes || kv_head_count <= 0 || kv_head_count > plan->params.hkv) {
+    fcp_set_error("fcp_plan_bwd_scratch_bytes: invalid argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  *bytes = bwd_scratch_need(plan, kv_head_count);
+  return FCP_OK;
+}
+
+extern "C" int fcp_attn_bwd_heads(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                                  const void* d_o, const float* lse, int32_t kv_head_begin, int32_t kv_head_count,
+                                  void* dq, void* dk, void* dv, void* scratch, int64_t scratch_bytes, void* stream) {
+  int rc = check_plan(plan);
+  if (rc != FCP_OK) return rc;
+  if (!q || !k || !v || !o || !d_o || !lse || !dq || !dk || !dv || !scratch) {
+    fcp_set_error("fcp_attn_bwd: NULL buffer");
+    return FCP_ERR_INVALID_ARG;
+  }
+  if (kv_head_begin < 0 || kv_head_count <= 0 || kv_head_begin + kv_head_count > plan->params.hkv) {
+    fcp_set_error("KV head range [%d, %d) outside [0, %d)", kv_head_begin, kv_head_begin + kv_head_count, plan->params.hkv);
+    return FCP_ERR_INVALID_ARG;
+  }
+  const int64_t need = bwd_scratch_need(plan, kv_head_count);
+  if (scratch_bytes < need) {
+    fcp_set_error("fcp_attn_bwd: scratch of %lld bytes, %lld needed", (long long)scratch_bytes, (long long)need);
+    return FCP_ERR_WORKSPACE;
+  }
+  const BwdTables tb{plan->d_bwd_units, plan->d_bwd_qranges, plan->d_bwd_work, plan->d_status, plan->d_status + 16,
+                     plan->sm_count};
+  return run_bwd(plan, tb, q, k, v, o, d_o, lse, kv_head_begin, kv_head_count, dq, dk, dv, scratch, plan,
+                 (cudaStream_t)stream);
+}
+
+extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, const void* v, const void* o,
+                            const void* d_o, const float* lse, void* dq, void* dk, void* dv, void* scratch,
+                            int64_t scratch_bytes, void* stream) {
+  if (!plan) {
+    fcp_set_error("plan is NULL");
+    return FCP_ERR_INVALID_ARG;
+  }
+  return fcp_attn_bwd_heads(plan, q, k, v, o, d_o, lse, 0, plan->params.hkv, dq, dk, dv, scratch, scratch_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -507,12 +586,11 @@ extern "C" int fcp_attn_bwd(const fcp_plan* plan, const void* q, const void* k, 
 // ---------------------------------------------------------------------------------------------
 namespace {
 struct HostLayout {
-  int64_t q, k, v, d_o, o, lse, dq, dk, dv, scratch, o_part, lse_part, total;
-  int heads_per_pass;
+  int64_t q, k, v, d_o, o, lse, dq, dk, dv, scratch, total;
 };
 inline int64_t al(int64_t x) { return (x + 255) / 256 * 256; }
 
-HostLayout host_layout(const fcp_plan* plan, int64_t limit_bytes) {
+HostLayout host_layout(const fcp_plan* plan) {
   const fcp_params& P = plan->params;
   const int64_t T = plan->T, D = P.head_dim;
   HostLayout L{};
@@ -527,18 +605,7 @@ HostLayout host_layout(const fcp_plan* plan, int64_t limit_bytes) {
   L.dq = take(T * P.hq * D * 2);
   L.dk = take(T * P.hkv * D * 2);
   L.dv = take(T * P.hkv * D * 2);
-  int64_t scratch = 0;
-  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
-  // the partial buffers are dead once merged, so they share memory with the backward scratch
-  const int64_t per_head = al(plan->R * D * 4) + al(plan->R * 4);
-  int hpp = P.hq;
-  if (limit_bytes > 0)
-    while (hpp > 1 && off + std::max<int64_t>(scratch, per_head * hpp) > limit_bytes) --hpp;
-  L.heads_per_pass = hpp;
-  L.scratch = off;
-  L.o_part = off;
-  L.lse_part = off + al(plan->R * hpp * D * 4);
-  off += al(std::max<int64_t>(scratch, al(plan->R * hpp * D * 4) + al(plan->R * hpp * 4)));
+  L.scratch = take(bwd_scratch_need(plan, P.hkv));
   L.total = off;
   return L;
 }
@@ -546,11 +613,7 @@ HostLayout host_layout(const fcp_plan* plan, int64_t limit_bytes) {
 
 extern "C" int fcp_host_workspace_bytes(const fcp_plan* plan, int64_t* bytes) {
   if (!plan || !bytes) return FCP_ERR_INVALID_ARG;
-  // smallest useful workspace: one head per pass would always fit, but prefer all heads when the
-  // partial buffers stay below 48 GiB
-  HostLayout L = host_layout(plan, 0);
-  if (L.total > (int64_t(96) << 30)) L = host_layout(plan, int64_t(96) << 30);
-  *bytes = L.total;
+  *bytes = host_layout(plan).total;
   return FCP_OK;
 }
 
@@ -558,6 +621,8 @@ namespace {
 // Cuts the batch into runs of consecutive sequences of about equal token counts (at most 8 runs, at
 // least about 8192 tokens each) and plans each run on its own: packed tensors are token-major, so a run
 // is one contiguous slice of every tensor and can be copied, computed and copied back independently.
+// Also creates the two copy streams and the events the host entry point orders its work with; all of
+// it belongs to the plan and is released by fcp_plan_destroy.
 int build_host_groups(const fcp_plan* plan, void* stream) {
   if (!plan->groups.empty()) return FCP_OK;
   const int B = plan->B;
@@ -570,6 +635,10 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
   }
   std::vector<fcp_plan*> groups;
   std::vector<int64_t> tok0;
+  auto fail = [&](int rc) {
+    for (fcp_plan* x : groups) fcp_plan_destroy(x);
+    return rc;
+  };
   int b0 = 0;
   for (int g = 0; g < want && b0 < B; ++g) {
     int b1 = b0 + 1;
@@ -584,18 +653,50 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
     if (rc == FCP_OK) rc = fcp_plan_upload(sub, stream);
     if (rc != FCP_OK) {
       if (sub) fcp_plan_destroy(sub);
-      for (fcp_plan* x : groups) fcp_plan_destroy(x);
-      return rc;
+      return fail(rc);
     }
     groups.push_back(sub);
     tok0.push_back(plan->cu_seqlens[b0]);
     b0 = b1;
   }
   tok0.push_back(T);
+  // streams and events: [0] start, [1] last copy out, then per group (inputs up, kernels done)
+  cudaStream_t in = nullptr, out = nullptr;
+  std::vector<void*> ev(2 + 2 * groups.size(), nullptr);
+  cudaError_t e = cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking);
+  for (size_t i = 0; i < ev.size() && e == cudaSuccess; ++i) {
+    cudaEvent_t x = nullptr;
+    e = cudaEventCreateWithFlags(&x, cudaEventDisableTiming);
+    ev[i] = x;
+  }
+  if (e != cudaSuccess) {
+    for (void* x : ev) if (x) cudaEventDestroy((cudaEvent_t)x);
+    if (in) cudaStreamDestroy(in);
+    if (out) cudaStreamDestroy(out);
+    fcp_set_error("fcp_attn_fwd_bwd_host: creating copy streams failed: %s", cudaGetErrorString(e));
+    return fail(FCP_ERR_CUDA);
+  }
+  plan->host_in = in;
+  plan->host_out = out;
+  plan->host_events = std::move(ev);
   plan->groups = std::move(groups);
   plan->group_tok0 = std::move(tok0);
   return FCP_OK;
 }
+
+// On any early exit of the host entry point: wait for the copies and kernels already queued, so that
+// nothing still writes into the caller's buffers after the call has returned an error.
+struct HostDrain {
+  cudaStream_t a, b, c;
+  bool armed = true;
+  ~HostDrain() {
+    if (!armed) return;
+    cudaStreamSynchronize(a);
+    cudaStreamSynchronize(b);
+    cudaStreamSynchronize(c);
+  }
+};
 }  // namespace
 
 extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, const void* k_host, const void* v_host,
@@ -608,7 +709,7 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
     fcp_set_error("fcp_attn_fwd_bwd_host: NULL buffer");
     return FCP_ERR_INVALID_ARG;
   }
-  const HostLayout L = host_layout(plan, workspace_bytes);
+  const HostLayout L = host_layout(plan);
   if (L.total > workspace_bytes) {
     fcp_set_error("fcp_attn_fwd_bwd_host: workspace of %lld bytes, %lld needed", (long long)workspace_bytes,
                   (long long)L.total);
@@ -624,77 +725,45 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   // Three streams: inputs of group g+1 come in and results of group g-1 go out while the kernels of
   // group g run on `stream`.  Everything is ordered after the work already queued on `stream` and is
   // complete when this call returns.
-  struct Side {
-    cudaStream_t in = nullptr, out = nullptr;
-    cudaEvent_t start = nullptr, last_out = nullptr;
-    std::vector<cudaEvent_t> up, done;
-    ~Side() {
-      for (cudaEvent_t e : up) if (e) cudaEventDestroy(e);
-      for (cudaEvent_t e : done) if (e) cudaEventDestroy(e);
-      if (start) cudaEventDestroy(start);
-      if (last_out) cudaEventDestroy(last_out);
-      if (in) cudaStreamDestroy(in);
-      if (out) cudaStreamDestroy(out);
-    }
-  } side;
-  FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.in, cudaStreamNonBlocking));
-  FCP_CUDA_CHECK(cudaStreamCreateWithFlags(&side.out, cudaStreamNonBlocking));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.start, cudaEventDisableTiming));
-  FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.last_out, cudaEventDisableTiming));
-  side.up.assign(G, nullptr);
-  side.done.assign(G, nullptr);
-  for (int g = 0; g < G; ++g) {
-    FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.up[g], cudaEventDisableTiming));
-    FCP_CUDA_CHECK(cudaEventCreateWithFlags(&side.done[g], cudaEventDisableTiming));
-  }
-  auto drain_sides = [&]() {
-    cudaStreamSynchronize(side.in);
-    cudaStreamSynchronize(side.out);
-    cudaStreamSynchronize(st);
-  };
-  FCP_CUDA_CHECK(cudaEventRecord(side.start, st));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.in, side.start, 0));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.start, 0));
+  cudaStream_t s_in = (cudaStream_t)plan->host_in, s_out = (cudaStream_t)plan->host_out;
+  auto EV = [&](int i) { return (cudaEvent_t)plan->host_events[i]; };
+  auto ev_up = [&](int g) { return EV(2 + 2 * g); };
+  auto ev_done = [&](int g) { return EV(3 + 2 * g); };
+  HostDrain drain{s_in, s_out, st};
+  FCP_CUDA_CHECK(cudaEventRecord(EV(0), st));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(s_in, EV(0), 0));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, EV(0), 0));
   for (int g = 0; g < G; ++g) {
     const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q + t0 * rq, (const char*)q_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, side.in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k + t0 * rkv, (const char*)k_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, side.in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v + t0 * rkv, (const char*)v_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, side.in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o + t0 * rq, (const char*)d_o_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, side.in));
-    FCP_CUDA_CHECK(cudaEventRecord(side.up[g], side.in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q + t0 * rq, (const char*)q_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k + t0 * rkv, (const char*)k_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v + t0 * rkv, (const char*)v_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o + t0 * rq, (const char*)d_o_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaEventRecord(ev_up(g), s_in));
   }
   for (int g = 0; g < G; ++g) {
     const fcp_plan* sub = plan->groups[g];
     const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.up[g], 0));
-    for (int h0 = 0; h0 < P.hq; h0 += L.heads_per_pass) {
-      const int hc = std::min(L.heads_per_pass, P.hq - h0);
-      if ((rc = fcp_attn_fwd_merged(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, h0, hc,
-                                    (float*)(w + L.o_part), (float*)(w + L.lse_part), w + L.o + t0 * rq,
-                                    (float*)(w + L.lse + t0 * rl), st)) != FCP_OK) {
-        drain_sides();
-        return rc;
-      }
-    }
-    int64_t scratch = 0;
-    fcp_plan_workspace_bytes(sub, 1, nullptr, nullptr, &scratch);
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_up(g), 0));
+    if ((rc = fcp_attn_fwd_fused(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, 0, P.hq, w + L.o + t0 * rq,
+                                 nullptr, (float*)(w + L.lse + t0 * rl), st)) != FCP_OK)
+      return rc;
     if ((rc = fcp_attn_bwd(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, w + L.o + t0 * rq,
                            w + L.d_o + t0 * rq, (float*)(w + L.lse + t0 * rl), w + L.dq + t0 * rq, w + L.dk + t0 * rkv,
-                           w + L.dv + t0 * rkv, w + L.scratch, scratch, st)) != FCP_OK) {
-      drain_sides();
+                           w + L.dv + t0 * rkv, w + L.scratch, bwd_scratch_need(sub, P.hkv), st)) != FCP_OK)
       return rc;
-    }
-    FCP_CUDA_CHECK(cudaEventRecord(side.done[g], st));
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(side.out, side.done[g], 0));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, side.out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, side.out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dq_host + t0 * rq, w + L.dq + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, side.out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dk_host + t0 * rkv, w + L.dk + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, side.out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dv_host + t0 * rkv, w + L.dv + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, side.out));
+    FCP_CUDA_CHECK(cudaEventRecord(ev_done(g), st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_done(g), 0));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dq_host + t0 * rq, w + L.dq + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dk_host + t0 * rkv, w + L.dk + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dv_host + t0 * rkv, w + L.dv + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));
   }
-  FCP_CUDA_CHECK(cudaEventRecord(side.last_out, side.out));
-  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, side.last_out, 0));
+  FCP_CUDA_CHECK(cudaEventRecord(EV(1), s_out));
+  FCP_CUDA_CHECK(cudaStreamWaitEvent(st, EV(1), 0));
   FCP_CUDA_CHECK(cudaStreamSynchronize(st));
+  drain.armed = false;
   return FCP_OK;
 }
 
@@ -749,9 +818,8 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
     fcp_set_error("fcp_attn_bwd_noalloc: NULL argument");
     return FCP_ERR_INVALID_ARG;
   }
-  int64_t need = 0, scratch = 0;
+  int64_t need = 0;
   fcp_noalloc_bytes_needed(plan, &need);
-  fcp_plan_workspace_bytes(plan, 1, nullptr, nullptr, &scratch);
   if (need > (int64_t)FCP_NOALLOC_MAX_BYTES) {
     fcp_set_error("fcp_attn_bwd_noalloc: this batch needs %lld bytes of scratch, the built-in arena holds %lld; "
                   "use fcp_attn_bwd with a caller-provided scratch buffer",
@@ -769,7 +837,6 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
   unsigned char* base = g_noalloc_ptr[dev];
   cudaStream_t st = (cudaStream_t)stream;
   const fcp_params& P = plan->params;
-  const int64_t T = plan->T, D = P.head_dim;
 
   // carve the arena: [status, counter | units | qranges | work | scratch]
   int64_t off = 256;
@@ -780,9 +847,8 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
   unsigned char* d_scratch = base + off;
 
   // the arena still holds the previous call's data: status, work counter and the dQ accumulator
-  // must start at zero; the tables are rewritten from the plan's host copy
+  // must start at zero (run_bwd clears the last two); the tables are rewritten from the plan's host copy
   FCP_CUDA_CHECK(cudaMemsetAsync(d_status, 0, 256, st));
-  FCP_CUDA_CHECK(cudaMemsetAsync(d_scratch, 0, (size_t)scratch, st));
   if (!plan->bwd_units.empty())
     FCP_CUDA_CHECK(cudaMemcpyAsync(d_units, plan->bwd_units.data(), plan->bwd_units.size() * 4, cudaMemcpyHostToDevice, st));
   if (!plan->bwd_qranges.empty())
@@ -790,57 +856,8 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
   if (!plan->bwd_work.empty())
     FCP_CUDA_CHECK(cudaMemcpyAsync(d_work, plan->bwd_work.data(), plan->bwd_work.size() * 4, cudaMemcpyHostToDevice, st));
 
-  const int64_t tpad = bwd_tpad(T);
-  float* dq_acc = (float*)d_scratch;
-  float* delta_t = dq_acc + T * P.hq * D;
-  float* lse2_t = delta_t + tpad * P.hq;
-  {
-    const int64_t rows = T * P.hq;
-    const int64_t blocks = (rows * (D / 8) + 255) / 256;
-    if (D == 128)
-      fcp_delta_kernel<128><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                              tpad, P.scale, delta_t, lse2_t);
-    else
-      fcp_delta_kernel<64><<<(unsigned)blocks, 256, 0, st>>>((const __nv_bfloat16*)o, (const __nv_bfloat16*)d_o, lse, T, P.hq,
-                                                             tpad, P.scale, delta_t, lse2_t);
-    FCP_CUDA_CHECK(cudaGetLastError());
-  }
-  CUtensorMap tq, tk, tv, tdo;
-  if ((rc = make_thd_map(&tq, q, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
-  if ((rc = make_thd_map(&tk, k, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
-  if ((rc = make_thd_map(&tv, v, T, P.hkv, (int)D, 128)) != FCP_OK) return rc;
-  if ((rc = make_thd_map(&tdo, d_o, T, P.hq, (int)D, 128)) != FCP_OK) return rc;
-  BwdArgs a;
-  a.units = d_units;
-  a.qranges = d_qranges;
-  a.work = d_work;
-  a.n_work = (int32_t)(plan->bwd_work.size() / 2);
-  a.counter = d_status + 16;
-  a.hq = P.hq;
-  a.hkv = P.hkv;
-  a.T = T;
-  a.t_stride = tpad;
-  a.scale = P.scale;
-  a.scale_log2 = P.scale * 1.4426950408889634f;
-  a.delta_t = delta_t;
-  a.lse2_t = lse2_t;
-  a.dq_acc = dq_acc;
-  a.dk = (__nv_bfloat16*)dk;
-  a.dv = (__nv_bfloat16*)dv;
-  a.status = d_status;
-  const int grid = (int)std::min<int64_t>(a.n_work, g_noalloc_sms[dev]);
-  if (grid > 0) {
-    if (D == 128)
-      fcp_bwd_kernel<128><<<grid, BWD_THREADS, BwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
-    else
-      fcp_bwd_kernel<64><<<grid, BWD_THREADS, BwdSmem<64>::DYN_BYTES, st>>>(tq, tk, tv, tdo, a);
-    FCP_CUDA_CHECK(cudaGetLastError());
-  }
-  const int64_t n8 = T * P.hq * D / 8;
-  const int blocks = (int)std::min<int64_t>((n8 + 255) / 256, (int64_t)g_noalloc_sms[dev] * 16);
-  fcp_dq_convert_kernel<<<blocks, 256, 0, st>>>(dq_acc, (__nv_bfloat16*)dq, n8);
-  FCP_CUDA_CHECK(cudaGetLastError());
-  return FCP_OK;
+  const BwdTables tb{d_units, d_qranges, d_work, d_status, d_status + 16, g_noalloc_sms[dev]};
+  return run_bwd(plan, tb, q, k, v, o, d_o, lse, 0, P.hkv, dq, dk, dv, d_scratch, nullptr, st);
 }
 
 extern "C" int fcp_noalloc_device_status(int32_t* status) {

@@ -345,51 +345,180 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
   p->fwd_units.reserve(fus.size() * FCP_FWD_UNIT_W);
   for (const FU& u : fus) p->fwd_units.insert(p->fwd_units.end(), u.f, u.f + FCP_FWD_UNIT_W);
 
-  // Backward: one unit per 128-key tile of every KV chunk; it visits the Q chunks of all block
-  // pairs whose kv_chunk is this chunk (q_chunk >= kv_chunk), the DIAG pair from its own tile on.
+  // Fused forward (merge on the fly): all items of a Q chunk run on one CTA, so the KV ranges of the
+  // chunk's block pairs are swept in one online softmax and no partial leaves the SM.  The ranges of
+  // a Q chunk are its pairs in kv_chunk order with adjacent FULL ranges joined.  In a causal plan
+  // that is the prefix [sequence start, chunk start) plus the DIAG range of the chunk itself, which
+  // one DIAG range starting at the sequence start describes exactly (every key before the chunk
+  // precedes every row of it); consecutive Q chunks of that form are joined into one run of rows,
+  // tiled in units of two Q tiles from the start of the run, so no tile is cut at a chunk edge.
+  struct Range { int32_t b, e, diag; };
+  std::vector<std::vector<Range>> q_cover(n_chunks_total);   // per Q chunk: joined KV ranges of its pairs
+  {
+    std::vector<std::vector<std::pair<int, int>>> by_q(n_chunks_total);   // (kv_chunk, kind)
+    for (const Pair& x : pairs) by_q[chunk_index0[x.seq] + x.qc].push_back({x.kc, x.kind});
+    for (int b = 0; b < B; ++b) {
+      const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+      for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
+        auto& v = by_q[chunk_index0[b] + c];
+        std::sort(v.begin(), v.end());
+        auto& out_r = q_cover[chunk_index0[b] + c];
+        for (auto& kk : v) {
+          const Range r{cbp[kk.first], cbp[kk.first + 1], kk.second};
+          if (!out_r.empty() && !out_r.back().diag && !r.diag && out_r.back().e == r.b) out_r.back().e = r.e;
+          else out_r.push_back(r);
+        }
+      }
+    }
+  }
+  {
+    std::vector<FU> gus;
+    auto emit_run = [&](int32_t t0, int32_t r0, int32_t r1) {     // rows [r0, r1) attend to [t0, row]
+      for (int32_t off = 0; off < r1 - r0; off += FCP_FWD_UNIT_ROWS) {
+        FU u{};
+        const int32_t rows = std::min<int32_t>(FCP_FWD_UNIT_ROWS, r1 - r0 - off);
+        u.f[FU_Q_ROW0] = r0 + off;
+        u.f[FU_Q_ROWS] = rows;
+        u.f[FU_N_RANGES] = 1;
+        u.f[FU_KV0_BEGIN] = t0; u.f[FU_KV0_END] = r1; u.f[FU_KV0_DIAG] = 1;
+        for (int s = 0; s < 2; ++s) {
+          const int32_t rs = std::min<int32_t>(FCP_TILE, rows - s * FCP_TILE);
+          u.f[FU_NT_STAGE0 + s] = rs > 0 ? ceil_div((int64_t)(r0 + off - t0) + s * FCP_TILE + rs, FCP_TILE) : 0;
+        }
+        u.f[FU_NT_RANGE0] = 0x7fffffff;
+        u.f[FU_ITEM] = -1;
+        u.f[FU_SINGLE_SLOT] = 1;
+        gus.push_back(u);
+      }
+    };
+    for (int b = 0; b < B; ++b) {
+      const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+      const int32_t t0 = cbp[0];
+      int32_t run0 = -1, run1 = -1;
+      for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
+        const int32_t q0 = cbp[c], q1 = cbp[c + 1];
+        if (q1 == q0) continue;
+        const auto& rg = q_cover[chunk_index0[b] + c];
+        const bool prefix = (rg.size() == 1 && rg[0].diag && rg[0].b == q0 && q0 == t0) ||
+                            (rg.size() == 2 && !rg[0].diag && rg[0].b == t0 && rg[0].e == q0 && rg[1].diag && rg[1].b == q0);
+        if (prefix) {
+          if (run0 < 0) run0 = q0;
+          else if (run1 != q0) { emit_run(t0, run0, run1); run0 = q0; }
+          run1 = q1;
+          continue;
+        }
+        if (run0 >= 0) { emit_run(t0, run0, run1); run0 = -1; }
+        // a chunk whose ranges are not a causal prefix keeps them as they are (at most two per unit)
+        if (rg.empty() || rg.size() > 2) {
+          delete p;
+          fcp_set_error("fcp_plan_blocks: Q chunk %d of sequence %d has %d disjoint KV ranges", c, b, (int)rg.size());
+          return FCP_ERR_UNSUPPORTED;
+        }
+        const int lastr = (int)rg.size() - 1;
+        const int nt_first = rg.size() == 2 ? ceil_div(rg[0].e - rg[0].b, FCP_TILE) : 0;
+        for (int32_t off = 0; off < q1 - q0; off += FCP_FWD_UNIT_ROWS) {
+          FU u{};
+          const int32_t rows = std::min<int32_t>(FCP_FWD_UNIT_ROWS, q1 - q0 - off);
+          u.f[FU_Q_ROW0] = q0 + off;
+          u.f[FU_Q_ROWS] = rows;
+          u.f[FU_N_RANGES] = (int32_t)rg.size();
+          u.f[FU_KV0_BEGIN] = rg[0].b; u.f[FU_KV0_END] = rg[0].e; u.f[FU_KV0_DIAG] = rg[0].diag;
+          if (rg.size() == 2) { u.f[FU_KV1_BEGIN] = rg[1].b; u.f[FU_KV1_END] = rg[1].e; u.f[FU_KV1_DIAG] = rg[1].diag; }
+          for (int s = 0; s < 2; ++s) {
+            const int32_t rs = std::min<int32_t>(FCP_TILE, rows - s * FCP_TILE);
+            int nt = 0;
+            if (rs > 0)
+              nt = nt_first + (rg[lastr].diag ? ceil_div((int64_t)(q0 + off - rg[lastr].b) + s * FCP_TILE + rs, FCP_TILE)
+                                              : ceil_div(rg[lastr].e - rg[lastr].b, FCP_TILE));
+            u.f[FU_NT_STAGE0 + s] = nt;
+          }
+          u.f[FU_NT_RANGE0] = rg.size() == 2 ? nt_first : 0x7fffffff;
+          u.f[FU_ITEM] = -1;
+          u.f[FU_SINGLE_SLOT] = 1;
+          gus.push_back(u);
+        }
+      }
+      if (run0 >= 0) emit_run(t0, run0, run1);
+    }
+    std::stable_sort(gus.begin(), gus.end(), [](const FU& a, const FU& b) {
+      return a.f[FU_NT_STAGE0] + a.f[FU_NT_STAGE1] > b.f[FU_NT_STAGE0] + b.f[FU_NT_STAGE1];
+    });
+    p->fused_units.reserve(gus.size() * FCP_FWD_UNIT_W);
+    for (const FU& u : gus) p->fused_units.insert(p->fused_units.end(), u.f, u.f + FCP_FWD_UNIT_W);
+  }
+
+  // Backward: one unit per 128-key tile; it visits the Q rows of all block pairs whose kv_chunk holds
+  // its keys (q_chunk >= kv_chunk), the DIAG pair from its own tile on.  The Q ranges of a KV chunk
+  // are its pairs in q_chunk order with adjacent ranges joined (a DIAG range followed by the FULL
+  // ranges of the later chunks is one DIAG range up to their end).  When every KV chunk of a sequence
+  // ends up with the single range [chunk start, sequence end) DIAG -- the causal plan -- the key
+  // tiles are cut from the start of the sequence instead of from each chunk start (a key tile may
+  // then span two KV chunks; the causal mask only depends on token positions), so that neither key
+  // tiles nor query tiles are cut at chunk edges.
   struct BU { int32_t f[FCP_BWD_UNIT_W]; };
   std::vector<BU> bus;
   {
-    // pairs grouped by (seq, kv_chunk), Q chunks ascending
     std::vector<std::vector<std::pair<int, int>>> by_kv(n_chunks_total);  // (q_chunk, kind)
     for (const Pair& x : pairs) by_kv[chunk_index0[x.seq] + x.kc].push_back({x.qc, x.kind});
     for (int b = 0; b < B; ++b) {
       const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
-      for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
+      const int nc = 2 * cp_degrees[b];
+      const int32_t t0 = cbp[0], t1 = cbp[nc];
+      std::vector<std::vector<Range>> kv_cover(nc);
+      bool causal_seq = true;
+      for (int c = 0; c < nc; ++c) {
         auto& v = by_kv[chunk_index0[b] + c];
-        if (v.empty()) continue;
         std::sort(v.begin(), v.end());
-        const int32_t first = (int32_t)(p->bwd_qranges.size() / FCP_BWD_QRANGE_W);
+        auto& out_r = kv_cover[c];
         for (auto& qk : v) {
-          const int32_t rowq[4] = {cbp[qk.first], cbp[qk.first + 1], qk.second, 0};
-          p->bwd_qranges.insert(p->bwd_qranges.end(), rowq, rowq + 4);
+          const Range r{cbp[qk.first], cbp[qk.first + 1], qk.second};
+          if (!out_r.empty() && !r.diag && out_r.back().e == r.b) out_r.back().e = r.e;   // keeps the first range's kind
+          else out_r.push_back(r);
         }
-        const int32_t k0 = cbp[c], k1 = cbp[c + 1];
+        if (cbp[c + 1] > cbp[c])
+          causal_seq = causal_seq && out_r.size() == 1 && out_r[0].diag && out_r[0].b == cbp[c] && out_r[0].e == t1;
+      }
+      auto emit_tiles = [&](int32_t k0, int32_t k1, int32_t first, const std::vector<Range>& rg) {
         for (int32_t off = 0, t = 0; off < k1 - k0; off += FCP_TILE, ++t) {
           BU u{};
           u.f[BU_KV_ROW0] = k0 + off;
           u.f[BU_KV_ROWS] = std::min<int32_t>(FCP_TILE, k1 - k0 - off);
           u.f[BU_FIRST_QRANGE] = first;
-          u.f[BU_N_QRANGES] = (int32_t)v.size();
+          u.f[BU_N_QRANGES] = (int32_t)rg.size();
           u.f[BU_KV_TILE] = t;
           int cost = 0;
-          for (auto& qk : v) {
-            const int nt = ceil_div(cbp[qk.first + 1] - cbp[qk.first], FCP_TILE);
-            cost += qk.second ? nt - t : nt;
+          for (const Range& r : rg) {
+            const int nt = ceil_div(r.e - r.b, FCP_TILE);
+            cost += r.diag ? std::max(0, nt - t) : nt;
           }
           u.f[BU_COST] = cost;
           u.f[BU_SEQ] = b;
           bus.push_back(u);
         }
+      };
+      auto push_ranges = [&](const std::vector<Range>& rg) {
+        const int32_t first = (int32_t)(p->bwd_qranges.size() / FCP_BWD_QRANGE_W);
+        for (const Range& r : rg) {
+          const int32_t rowq[4] = {r.b, r.e, r.diag, 0};
+          p->bwd_qranges.insert(p->bwd_qranges.end(), rowq, rowq + 4);
+        }
+        return first;
+      };
+      if (causal_seq) {
+        const std::vector<Range> whole{Range{t0, t1, 1}};
+        emit_tiles(t0, t1, push_ranges(whole), whole);
+      } else {
+        for (int c = 0; c < nc; ++c)
+          if (!kv_cover[c].empty()) emit_tiles(cbp[c], cbp[c + 1], push_ranges(kv_cover[c]), kv_cover[c]);
       }
     }
   }
   for (const BU& u : bus) p->bwd_units.insert(p->bwd_units.end(), u.f, u.f + FCP_BWD_UNIT_W);
-  // Execution order of the backward work items (unit, KV head).  dQ is accumulated with fp32
-  // reductions in global memory, which only run at L2 speed while the rows they touch stay
-  // resident: so all CTAs work on one (sequence, KV head) panel at a time, key tiles in ascending
-  // position (descending cost), and sweep the query tiles roughly in step.  Sequences go longest
-  // first, which leaves the small units for the tail of the schedule.
+  // Execution order of the backward units within one KV head (the kernel runs the KV heads one after
+  // the other, each over this list).  dQ is accumulated with fp32 reductions in global memory, which
+  // only run at L2 speed while the rows they touch stay resident: so all CTAs work on one
+  // (sequence, KV head) panel at a time, key tiles in ascending position (descending cost), and
+  // sweep the query tiles roughly in step.  Sequences go longest first.
   {
     std::vector<int> seq_order(B);
     std::iota(seq_order.begin(), seq_order.end(), 0);
@@ -397,11 +526,7 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
     std::vector<std::vector<int32_t>> units_of(B);
     for (size_t i = 0; i < bus.size(); ++i) units_of[bus[i].f[BU_SEQ]].push_back((int32_t)i);   // ascending key position
     for (int b : seq_order)
-      for (int hk = 0; hk < params->hkv; ++hk)
-        for (int32_t u : units_of[b]) {
-          p->bwd_work.push_back(u);
-          p->bwd_work.push_back(hk);
-        }
+      for (int32_t u : units_of[b]) p->bwd_work.push_back(u);
   }
 
   // Merge: runs of up to FCP_MERGE_TOKENS tokens inside one chunk.  Chunks with two or more slots
@@ -442,6 +567,7 @@ extern "C" int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t**
     case FCP_TABLE_BWD_QRANGES: v = &plan->bwd_qranges; break;
     case FCP_TABLE_MERGE_UNITS: v = &plan->merge_units; break;
     case FCP_TABLE_BWD_WORK: v = &plan->bwd_work; break;
+    case FCP_TABLE_FUSED_UNITS: v = &plan->fused_units; break;
     default: fcp_set_error("fcp_plan_get: unknown table %d", which); return FCP_ERR_INVALID_ARG;
   }
   *host_ptr = v->data();
@@ -461,6 +587,7 @@ extern "C" int fcp_plan_info(const fcp_plan* plan, int32_t which, int64_t* value
     case 6: *value = (int64_t)plan->merge_units.size() / FCP_MERGE_UNIT_W; break;
     case 7: *value = plan->B; break;
     case 8: *value = plan->n_merge_multi; break;
+    case 9: *value = (int64_t)plan->fused_units.size() / FCP_FWD_UNIT_W; break;
     default: return FCP_ERR_INVALID_ARG;
   }
   return FCP_OK;

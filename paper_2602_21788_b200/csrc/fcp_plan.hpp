@@ -31,7 +31,7 @@ struct fcp_plan {
   int64_t R = 0;   // rows of the partial buffers
   int32_t n_merge_multi = 0;   // merge units of chunks with two or more slots (they come first in merge_units)
   std::vector<int32_t> cu_seqlens, chunk_offset, chunk_bounds, pairs, items, slot_offset, slot_rows;
-  std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units, bwd_work;
+  std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units, bwd_work, fused_units;
 
   // device copy (fcp_plan_upload)
   int device = -1;
@@ -41,6 +41,7 @@ struct fcp_plan {
   int32_t* d_bwd_qranges = nullptr;
   int32_t* d_merge_units = nullptr;
   int32_t* d_bwd_work = nullptr;
+  int32_t* d_fused_units = nullptr;
   int32_t* d_slot_offset = nullptr;
   int32_t* d_slot_rows = nullptr;
   int32_t* d_status = nullptr; // [4]: status word, diagnostic
@@ -50,6 +51,9 @@ struct fcp_plan {
   // entry point, which pipelines copies and kernels over them (owned by this plan).
   mutable std::vector<fcp_plan*> groups;
   mutable std::vector<int64_t> group_tok0;   // first packed token of each group, plus T at the end
+  mutable void* host_in = nullptr;           // cudaStream_t: host -> device copies of the host entry point
+  mutable void* host_out = nullptr;          // cudaStream_t: device -> host copies
+  mutable std::vector<void*> host_events;    // cudaEvent_t: start, last copy out, then (inputs up, kernels done) per group
 
   // optional kernel timing: ring of event pairs per kernel kind (void* = cudaEvent_t)
   bool profiling = false;

@@ -19,12 +19,14 @@ FCP_ERR_CUDA, FCP_ERR_TIMEOUT, FCP_ERR_NOT_UPLOADED = -5, -6, -7
 FCP_MAX_DEGREE = 64
 
 TABLES = dict(cu_seqlens=0, chunk_offset=1, chunk_bounds=2, pairs=3, items=4, slot_offset=5, slot_rows=6,
-              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11)
-_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, bwd_work=2)
-INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7, n_merge_multi=8)
+              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11, fused_units=12)
+_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, fused_units=16)
+INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7, n_merge_multi=8,
+            n_fused_units=9)
 
 EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
-           "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_attn_fwd_merged", "fcp_lse_merge", "fcp_attn_bwd",
+           "fcp_plan_bwd_scratch_bytes", "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_attn_fwd_merged",
+           "fcp_attn_fwd_fused", "fcp_lse_merge", "fcp_attn_bwd", "fcp_attn_bwd_heads",
            "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
            "fcp_plan_kernel_ms", "fcp_noalloc_bytes_needed", "fcp_attn_bwd_noalloc", "fcp_noalloc_device_status",
            "fcp_status_string",
@@ -73,6 +75,9 @@ def lib() -> C.CDLL:
     L.fcp_plan_set_profiling.argtypes = [vp, C.c_int32]
     L.fcp_plan_kernel_ms.argtypes = [vp, C.c_int32, i32p, f32p]
     L.fcp_attn_bwd.argtypes = [vp] * 11 + [C.c_int64, vp]
+    L.fcp_attn_bwd_heads.argtypes = [vp] * 7 + [C.c_int32, C.c_int32] + [vp] * 4 + [C.c_int64, vp]
+    L.fcp_attn_fwd_fused.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, vp, vp, vp, vp]
+    L.fcp_plan_bwd_scratch_bytes.argtypes = [vp, C.c_int32, i64p]
     L.fcp_host_workspace_bytes.argtypes = [vp, i64p]
     L.fcp_attn_fwd_bwd_host.argtypes = [vp] * 11 + [C.c_int64, vp]
     L.fcp_last_device_status.argtypes = [vp, i32p]
@@ -168,6 +173,11 @@ class Plan:
         _check(lib().fcp_plan_workspace_bytes(self.handle, int(heads_per_pass or self.hq), C.byref(a), C.byref(b), C.byref(c)))
         return a.value, b.value, c.value
 
+    def bwd_scratch_bytes(self, kv_head_count=None) -> int:
+        v = C.c_int64(0)
+        _check(lib().fcp_plan_bwd_scratch_bytes(self.handle, int(kv_head_count or self.hkv), C.byref(v)))
+        return v.value
+
     def host_workspace_bytes(self) -> int:
         v = C.c_int64(0)
         _check(lib().fcp_host_workspace_bytes(self.handle, C.byref(v)))
@@ -208,6 +218,12 @@ def fcp_attn_fwd_merged(plan: Plan, q, k, v, o_partial, lse_partial, o, lse, hea
                                      _ptr(lse_partial), _ptr(o), _ptr(lse), C.c_void_p(stream)))
 
 
+def fcp_attn_fwd_fused(plan: Plan, q, k, v, o, lse, head_begin=0, head_count=None, stream=0, o_f32=None):
+    hc = plan.hq - head_begin if head_count is None else head_count
+    _check(lib().fcp_attn_fwd_fused(plan.handle, _ptr(q), _ptr(k), _ptr(v), int(head_begin), int(hc), _ptr(o), _ptr(o_f32),
+                                    _ptr(lse), C.c_void_p(stream)))
+
+
 def fcp_lse_merge(plan: Plan, o_partial, lse_partial, o, lse, head_begin=0, head_count=None, stream=0, o_f32=None):
     hc = plan.hq - head_begin if head_count is None else head_count
     _check(lib().fcp_lse_merge(plan.handle, _ptr(o_partial), _ptr(lse_partial), int(head_begin), int(hc), _ptr(o),
@@ -217,6 +233,13 @@ def fcp_lse_merge(plan: Plan, o_partial, lse_partial, o, lse, head_begin=0, head
 def fcp_attn_bwd(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, scratch, scratch_bytes, stream=0):
     _check(lib().fcp_attn_bwd(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), _ptr(dq), _ptr(dk),
                               _ptr(dv), _ptr(scratch), int(scratch_bytes), C.c_void_p(stream)))
+
+
+def fcp_attn_bwd_heads(plan: Plan, q, k, v, o, d_o, lse, kv_head_begin, kv_head_count, dq, dk, dv, scratch, scratch_bytes,
+                       stream=0):
+    _check(lib().fcp_attn_bwd_heads(plan.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(d_o), _ptr(lse), int(kv_head_begin),
+                                    int(kv_head_count), _ptr(dq), _ptr(dk), _ptr(dv), _ptr(scratch), int(scratch_bytes),
+                                    C.c_void_p(stream)))
 
 
 def fcp_attn_fwd_bwd_host(plan: Plan, q, k, v, d_o, o, lse, dq, dk, dv, workspace, workspace_bytes, stream=0):

@@ -21,17 +21,22 @@ def bf16_dev_to_f64(t: torch.Tensor) -> np.ndarray:
 class DeviceState:
     """All device buffers of one workload (inputs, partials, outputs, scratch) and its uploaded plan."""
 
-    def __init__(self, w: synth.Workload, q, k, v, do=None, heads_per_pass=None, want_o_f32=False):
+    def __init__(self, w: synth.Workload, q, k, v, do=None, heads_per_pass=None, want_o_f32=False, partials=True,
+                 kv_heads_per_bwd_pass=None):
+        """q, k, v, do: bf16 bit patterns on the host (numpy uint16) or bf16 tensors already on the device.
+        `partials=False` skips the partial buffers (enough for the fused forward)."""
         self.w = w
         self.plan = fcp.fcp_plan_blocks(w.seqlens, w.cp_degrees, w.hq, w.hkv, w.head_dim).upload()
         T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
         self.hpp = heads_per_pass or hq
-        self.q, self.k, self.v = to_dev_bf16(q), to_dev_bf16(k), to_dev_bf16(v)
-        self.do = to_dev_bf16(do) if do is not None else None
+        dev = lambda a: a if isinstance(a, torch.Tensor) else to_dev_bf16(a)
+        self.q, self.k, self.v = dev(q), dev(k), dev(v)
+        self.do = dev(do) if do is not None else None
         R = self.plan.info("R")
         self.R = R
-        self.o_part = torch.empty((R, self.hpp, D), dtype=torch.float32, device="cuda")
-        self.lse_part = torch.empty((R, self.hpp), dtype=torch.float32, device="cuda")
+        if partials:
+            self.o_part = torch.empty((R, self.hpp, D), dtype=torch.float32, device="cuda")
+            self.lse_part = torch.empty((R, self.hpp), dtype=torch.float32, device="cuda")
         self.o = torch.empty((T, hq, D), dtype=torch.bfloat16, device="cuda")
         self.lse = torch.empty((T, hq), dtype=torch.float32, device="cuda")
         self.o_f32 = torch.empty((T, hq, D), dtype=torch.float32, device="cuda") if want_o_f32 else None
@@ -39,7 +44,8 @@ class DeviceState:
             self.dq = torch.empty((T, hq, D), dtype=torch.bfloat16, device="cuda")
             self.dk = torch.empty((T, hkv, D), dtype=torch.bfloat16, device="cuda")
             self.dv = torch.empty((T, hkv, D), dtype=torch.bfloat16, device="cuda")
-            self.scratch_bytes = self.plan.workspace_bytes(1)[2]
+            self.kv_pass = kv_heads_per_bwd_pass or hkv
+            self.scratch_bytes = self.plan.bwd_scratch_bytes(self.kv_pass)
             self.scratch = torch.empty(self.scratch_bytes, dtype=torch.uint8, device="cuda")
 
     def forward(self, stream=None, merged=False):
@@ -55,10 +61,23 @@ class DeviceState:
                 fcp.fcp_attn_fwd(self.plan, self.q, self.k, self.v, self.o_part, self.lse_part, h0, hc, st)
                 fcp.fcp_lse_merge(self.plan, self.o_part, self.lse_part, self.o, self.lse, h0, hc, st, o_f32=self.o_f32)
 
+    def forward_fused(self, stream=None):
+        """Forward with the merge on the fly (no partial buffers), in head passes of `heads_per_pass`."""
+        st = (stream or torch.cuda.current_stream()).cuda_stream
+        for h0 in range(0, self.w.hq, self.hpp):
+            hc = min(self.hpp, self.w.hq - h0)
+            fcp.fcp_attn_fwd_fused(self.plan, self.q, self.k, self.v, self.o, self.lse, h0, hc, st, o_f32=self.o_f32)
+
     def backward(self, stream=None):
         st = (stream or torch.cuda.current_stream()).cuda_stream
-        fcp.fcp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
-                         self.scratch, self.scratch_bytes, st)
+        if self.kv_pass == self.w.hkv:
+            fcp.fcp_attn_bwd(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, self.dq, self.dk, self.dv,
+                             self.scratch, self.scratch_bytes, st)
+            return
+        for k0 in range(0, self.w.hkv, self.kv_pass):
+            kc = min(self.kv_pass, self.w.hkv - k0)
+            fcp.fcp_attn_bwd_heads(self.plan, self.q, self.k, self.v, self.o, self.do, self.lse, k0, kc, self.dq, self.dk,
+                                   self.dv, self.scratch, self.scratch_bytes, st)
 
     def check_status(self):
         st = self.plan.device_status()
@@ -66,9 +85,15 @@ class DeviceState:
             raise RuntimeError(f"device status {fcp.status_string(int(st[0]))}: where={st[1]} block={st[2]} thread={st[3]}")
 
 
-def run_fwd_bwd(w, q, k, v, do=None, heads_per_pass=None, keep_partials=False, want_o_f32=True):
-    ds = DeviceState(w, q, k, v, do, heads_per_pass, want_o_f32)
-    ds.forward()
+def run_fwd_bwd(w, q, k, v, do=None, heads_per_pass=None, keep_partials=False, want_o_f32=True, fused=False,
+                kv_heads_per_bwd_pass=None):
+    """`fused`: forward through fcp_attn_fwd_fused instead of fcp_attn_fwd + fcp_lse_merge."""
+    ds = DeviceState(w, q, k, v, do, heads_per_pass, want_o_f32, partials=not fused,
+                     kv_heads_per_bwd_pass=kv_heads_per_bwd_pass)
+    if fused:
+        ds.forward_fused()
+    else:
+        ds.forward()
     out = {}
     if do is not None:
         ds.backward()

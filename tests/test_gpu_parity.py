@@ -118,6 +118,71 @@ def test_reduced_workloads(name):
     _check_full(w)
 
 
+def _check_fused(w, heads_per_pass=None):
+    """fcp_attn_fwd_fused (merge on the fly, no partials) against the fp64 oracle, and against the
+    partial-producing path of the same plan."""
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    q, k, v = w.tensors(with_do=False)
+    res = run_fwd_bwd(w, q, k, v, None, heads_per_pass=heads_per_pass, fused=True)
+    o_ref, lse_ref = A.attention_fwd_packed(f64(q), f64(k), f64(v), w.cu_seqlens)
+    e = np.abs(res["o_f32"] - o_ref)
+    assert e.max() <= O_MAX and e.mean() <= O_MEAN, (e.max(), e.mean())
+    eb = np.abs(res["o"] - o_ref)
+    assert np.all(eb <= O_MAX + np.abs(o_ref) * 2.0 ** -8) and eb.mean() <= O_MEAN, (eb.max(), eb.mean())
+    assert np.abs(res["lse"] - lse_ref).max() <= LSE_MAX
+    part = run_fwd_bwd(w, q, k, v, None, heads_per_pass=heads_per_pass)
+    assert np.abs(part["o_f32"] - res["o_f32"]).max() <= O_MAX and np.abs(part["lse"] - res["lse"]).max() <= LSE_MAX
+
+
+@pytest.mark.parametrize("lens,degs,hq,hkv,D", EDGE_CASES)
+def test_fused_forward_edge_shapes(lens, degs, hq, hkv, D):
+    _check_fused(_wl(lens, degs, hq, hkv, D, seed=3))
+
+
+@pytest.mark.parametrize("name", ["tiny", "llama8b_64k", "longtail_256k", "bimodal_128k", "extreme_512k"])
+def test_fused_forward_workloads(name):
+    w = synth.make_workload(name, 0)
+    _check_fused(w if name == "tiny" else synth.reduced(w), heads_per_pass=3 if name == "bimodal_128k" else None)
+
+
+def test_fused_forward_is_bitwise_reproducible_and_independent_of_the_degrees():
+    """One CTA sweeps a row's keys in position order whatever the plan's degrees, so the fused forward of
+    the configured degrees and of all d = 1 give the same bits."""
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = synth.reduced(synth.make_workload("bimodal_128k", 1), len_div=8)
+    q, k, v = w.tensors(with_do=False)
+    a = run_fwd_bwd(w, q, k, v, None, fused=True)
+    b = run_fwd_bwd(w, q, k, v, None, fused=True)
+    assert np.array_equal(a["o"], b["o"]) and np.array_equal(a["lse"], b["lse"])
+    w1 = _wl(w.seqlens, np.ones_like(w.cp_degrees), w.hq, w.hkv, w.head_dim, seed=w.seed)
+    c = run_fwd_bwd(w1, q, k, v, None, fused=True)
+    assert np.array_equal(a["o"], c["o"]) and np.array_equal(a["lse"], c["lse"])
+
+
+def test_backward_in_kv_head_passes_gives_the_same_result():
+    """fcp_attn_bwd_heads over disjoint KV-head ranges == fcp_attn_bwd over all heads: dK/dV bit for bit
+    (no sum crosses KV heads, no atomics), dQ to the order of its fp32 reductions."""
+    from paper_2602_21788_b200 import fcp
+    from paper_2602_21788_b200.runner import run_fwd_bwd
+    w = _wl([700, 300, 129], [3, 2, 1], 8, 4, 128, seed=5)
+    q, k, v, do = w.tensors()
+    a = run_fwd_bwd(w, q, k, v, do)
+    b = run_fwd_bwd(w, q, k, v, do, kv_heads_per_bwd_pass=3)      # passes of 3 + 1 KV heads
+    assert np.array_equal(a["dk"], b["dk"]) and np.array_equal(a["dv"], b["dv"])
+    assert np.linalg.norm(a["dq"] - b["dq"]) <= 1e-2 * np.linalg.norm(a["dq"])
+    dq_ref, dk_ref, dv_ref = A.attention_bwd_packed(f64(q), f64(k), f64(v), f64(do), w.cu_seqlens)
+    for name, ref in (("dq", dq_ref), ("dk", dk_ref), ("dv", dv_ref)):
+        ok, rel = _grad_ok(b[name], ref)
+        assert ok, (name, rel)
+    ds = b["state"]
+    assert ds.plan.bwd_scratch_bytes(3) < ds.plan.bwd_scratch_bytes(4) == ds.plan.workspace_bytes(1)[2]
+    with pytest.raises(fcp.FcpError) as e:
+        fcp.fcp_attn_bwd_heads(ds.plan, ds.q, ds.k, ds.v, ds.o, ds.do, ds.lse, 3, 2, ds.dq, ds.dk, ds.dv, ds.scratch,
+                               ds.scratch_bytes, 0)
+    assert e.value.status == fcp.FCP_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+
+
 def test_head_passes_give_the_same_result():
     from paper_2602_21788_b200.runner import run_fwd_bwd
     w = _wl([700, 300], [3, 2], 8, 2, 128, seed=5)

@@ -58,12 +58,10 @@ def test_block_plan_bit_exact_on_workloads(name, seed):
     assert plan.info("T") == w.total_tokens
 
 
-def _cover(plan, lens):
-    """Token-pair coverage implied by the derived forward and backward work lists."""
-    cu = np.concatenate([[0], np.cumsum(lens)])
-    T = int(cu[-1])
+def _cover_fwd(units, T):
+    """Token-pair coverage implied by a table of forward work units (per-item or fused)."""
     fwd = np.zeros((T, T), dtype=np.int32)
-    for u in plan.table("fwd_units"):
+    for u in units:
         q0, rows, prow, nr = u[0], u[1], u[2], u[3]
         nts = [u[10], u[11]]
         nr0 = u[12]
@@ -80,6 +78,14 @@ def _cover(plan, lens):
                     limit = min(limit, 128)
                     assert limit >= 1
                     fwd[qp, ks:ks + limit] += 1
+    return fwd
+
+
+def _cover(plan, lens):
+    """Token-pair coverage implied by the derived forward and backward work lists."""
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    T = int(cu[-1])
+    fwd = _cover_fwd(plan.table("fwd_units"), T)
     bwd = np.zeros((T, T), dtype=np.int32)
     qr = plan.table("bwd_qranges")
     for u in plan.table("bwd_units"):
@@ -104,12 +110,37 @@ def _cover(plan, lens):
     return fwd, bwd, want
 
 
-@pytest.mark.parametrize("lens,degs", [([300, 5, 129], [1, 3, 2]), ([700], [2]), ([1030], [3]), ([257, 256, 255], [1, 1, 1])])
+def _pairs_cover(plan, lens):
+    """Token-pair coverage of the canonical block pairs themselves (FULL: whole block, DIAG: its triangle)."""
+    T = int(sum(lens))
+    cb, co = plan.table("chunk_bounds"), plan.table("chunk_offset")
+    out = np.zeros((T, T), dtype=np.int32)
+    for (b, r, s, qc, kc, kind) in plan.table("pairs"):
+        q0, q1, k0, k1 = cb[co[b] + qc], cb[co[b] + qc + 1], cb[co[b] + kc], cb[co[b] + kc + 1]
+        blk = np.ones((q1 - q0, k1 - k0), dtype=np.int32)
+        out[q0:q1, k0:k1] += np.tril(blk) if kind else blk
+    return out
+
+
+@pytest.mark.parametrize("lens,degs", [([300, 5, 129], [1, 3, 2]), ([700], [2]), ([1030], [3]), ([257, 256, 255], [1, 1, 1]),
+                                       ([3, 1000, 2], [4, 7, 1]), ([513], [64])])
 def test_work_lists_cover_the_causal_triangle_exactly_once(lens, degs):
     plan = fcp.fcp_plan_blocks(lens, degs, 4, 4, 64)
     fwd, bwd, want = _cover(plan, lens)
     assert np.array_equal(fwd, want)
     assert np.array_equal(bwd, want)
+    # the fused forward units (all items of a Q chunk on one CTA) execute the same token pairs as the
+    # plan's block pairs, each exactly once, and every query row belongs to exactly one unit
+    pairs = _pairs_cover(plan, lens)
+    assert np.array_equal(pairs, want)
+    fused_units = plan.table("fused_units")
+    assert np.array_equal(_cover_fwd(fused_units, int(sum(lens))), pairs)
+    rows = np.zeros(sum(lens), dtype=np.int32)
+    for u in fused_units:
+        rows[u[0]:u[0] + u[1]] += 1
+    assert np.all(rows == 1) and plan.info("n_fused_units") == len(fused_units)
+    # backward execution order: a permutation of the units
+    assert sorted(plan.table("bwd_work").tolist()) == list(range(plan.info("n_bwd_units")))
     # every partial row is written by exactly one forward unit
     R = plan.info("R")
     hit = np.zeros(R, dtype=np.int32)
