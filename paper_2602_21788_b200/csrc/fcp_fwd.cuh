@@ -47,6 +47,8 @@ struct FwdArgs {
   const int32_t* units;   // [n_units][16]
   int32_t n_units;
   int32_t head_begin, head_count, hq, hkv;
+  int32_t head_group;     // heads that are adjacent in the work order: hq/hkv when the head range is made of whole
+                          // KV-head groups, else 1; head_count % head_group == 0
   float scale_log2;       // softmax scale * log2(e)
   float* o_partial;       // [R][head_count][D]
   float* lse_partial;     // [R][head_count]
@@ -113,6 +115,23 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   const int64_t n_work = (int64_t)a.n_units * a.head_count;
   const int g = a.hq / a.hkv;
+  // Work item w = (head within an inner group of `gi` heads, unit, group), innermost first: with gi =
+  // the query heads of one KV head, the CTAs that run at the same time work on adjacent units of the
+  // same KV head and stream the same K/V tiles (one copy in L2 serves them all).  CTA c takes the
+  // items c, 2G-1-c, 2G+c, ... (G = grid size): units are sorted by cost, so alternating the
+  // direction of every other round evens out the systematic bias of a fixed stride.  Every role
+  // walks the same sequence.
+  const int gi = a.head_group;
+  auto work_item = [&](int64_t round, const int32_t*& U, int& h) -> bool {
+    const int64_t G = gridDim.x;
+    const int64_t w = round * G + ((round & 1) ? G - 1 - (int64_t)blockIdx.x : (int64_t)blockIdx.x);
+    if (w >= n_work) return false;          // only in the last round
+    const int64_t grp = w / gi;
+    U = a.units + (size_t)(grp % a.n_units) * FCP_FWD_UNIT_W;
+    h = a.head_begin + (int)(grp / a.n_units) * gi + (int)(w % gi);
+    return true;
+  };
+  const int64_t n_rounds = (n_work + gridDim.x - 1) / gridDim.x;
 
   if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_CTRL ";");
   if (warp == 0) {
@@ -121,9 +140,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       uint32_t kv_it = 0, qcnt[2] = {0, 0};
       bool ok = true;
 #pragma unroll 1
-      for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-        const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
-        const int h = a.head_begin + (int)(w % a.head_count);
+      for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+        const int32_t* U;
+        int h;
+        if (!work_item(rnd, U, h)) continue;
         const int hk = h / g;
         const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
         const int q_row0 = __ldg(U + FU_Q_ROW0);
@@ -176,8 +196,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       uint32_t kv_it = 0, qcnt = 0, pcnt = 0, ocnt = 0;
       bool ok = true;
 #pragma unroll 1
-      for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-        const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+      for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+        const int32_t* U;
+        int h;
+        if (!work_item(rnd, U, h)) continue;
         const int nts = __ldg(U + FU_NT_STAGE0 + s);
         const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
         if (nts > 0) {
@@ -235,8 +257,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     uint32_t scnt = 0, ucnt = 0, tcnt = 0;
     bool ok = true;
 #pragma unroll 1
-    for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-      const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
+    for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+      const int32_t* U;
+      int h;
+      if (!work_item(rnd, U, h)) continue;
       const int nts = __ldg(U + FU_NT_STAGE0 + s);
       const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
       const int q_pos = __ldg(U + FU_Q_ROW0) + s * 128 + row;
@@ -362,9 +386,11 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     uint32_t ecnt0 = 0, ecnt1 = 0;             // phases seen per Q tile
     bool ok = true;
 #pragma unroll 1
-    for (int64_t w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
-      const int32_t* U = a.units + (size_t)(w / a.head_count) * FCP_FWD_UNIT_W;
-      const int hl = (int)(w % a.head_count);
+    for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+      const int32_t* U;
+      int h;
+      if (!work_item(rnd, U, h)) continue;
+      const int hl = h - a.head_begin;
       const int q_rows = __ldg(U + FU_Q_ROWS);
       const int64_t prow0 = (int64_t)__ldg(U + FU_PART_ROW0);
       // A Q chunk with one slot has nothing to merge: its partial is the result, and goes straight to

@@ -374,6 +374,10 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
   a.head_count = head_count;
   a.hq = P.hq;
   a.hkv = P.hkv;
+  {
+    const int g = P.hq / P.hkv;
+    a.head_group = (head_begin % g == 0 && head_count % g == 0) ? g : 1;
+  }
   a.scale_log2 = P.scale * 1.4426950408889634f;
   a.o_partial = o_partial;
   a.lse_partial = lse_partial;
