@@ -194,16 +194,6 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
-def device_inputs(w, seed):
-    """q, k, v, dO ~ N(0,1) as bf16 device tensors from a seeded device generator."""
-    import torch
-    g = torch.Generator(device="cuda")
-    g.manual_seed(0xFC9 + 7919 * int(seed))
-    T, D = w.total_tokens, w.head_dim
-    mk = lambda h: torch.randn((T, h, D), dtype=torch.bfloat16, device="cuda", generator=g)
-    return mk(w.hq), mk(w.hkv), mk(w.hkv), mk(w.hq)
-
-
 def time_planner(w, reps=20):
     """Host time of the two planner calls alone (no CUDA call inside the timers), microseconds."""
     from paper_2602_21788_b200 import costfit, fcp
@@ -242,7 +232,7 @@ def measure(w, seed, steps, warmup, sampler, dist_ctx, heads_per_pass=0, want_pa
     from paper_2602_21788_b200 import ranks
     from paper_2602_21788_b200.runner import DeviceState
 
-    q, k, v, do = device_inputs(w, seed)
+    q, k, v, do = w.device_tensors()
     ds = DeviceState(w, q, k, v, do, heads_per_pass=heads_per_pass or None, partials=False)
     del q, k, v, do
     plan = ds.plan

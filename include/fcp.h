@@ -288,6 +288,16 @@ int fcp_noalloc_device_status(int32_t* status);
 int fcp_plan_set_profiling(fcp_plan* plan, int32_t enable);
 int fcp_plan_kernel_ms(const fcp_plan* plan, int32_t kind, int32_t* launches, float* mean_ms);
 
+/* fcp_selftest_bounded_wait — device.  Every wait inside the persistent kernels (on an mbarrier fed
+ * by TMA, the tensor core or another warp) is bounded: after 2 s without progress the waiter gives
+ * up, the CTA unwinds, and FCP_ERR_TIMEOUT appears in the status words instead of a hung GPU.  This
+ * call exercises exactly that code on purpose and safely: one warp waits on a barrier nobody
+ * arrives at, with the limit set to `limit_us` microseconds (1..100000), so the launch ends by
+ * itself after about that long.  Writes the four status words the wait produced to the host array
+ * status[4]: {FCP_ERR_TIMEOUT, 901 (the code of the wait site), CTA index 0, 0}.  Uses status words
+ * of its own (no plan is involved or marked).  Synchronises `stream`.                             */
+int fcp_selftest_bounded_wait(uint32_t limit_us, int32_t* status, void* stream);
+
 const char* fcp_status_string(int status);
 const char* fcp_last_error_message(void);
 

@@ -104,6 +104,44 @@ def plan_blocks(seqlens, cp_degrees):
                 chunk_slots=chunk_slots, n_partial_rows=row)
 
 
+def span_tables(seqlens, cp_degrees, spans_per_seq):
+    """Integer tables of a plan whose sequences carry bidirectional spans (a query inside a span
+    [a, b) also sees the later keys of its span; Sec. 4.3 motivates the mask efficiency factor eta
+    with such tokens).  Positions in `spans_per_seq` are sequence-relative; the tables are packed.
+
+    row_limit[t]   : first key (packed index) that query t does not see: t + 1, or its span's end
+    first_query[t] : first query (packed index) that sees key t: t, or its span's begin
+    span_pairs     : (seq, rank, step, q_chunk, kv_chunk) with kv_chunk > q_chunk, sorted: the block
+                     pairs above the chunk diagonal in which some query sees some key.  The ring
+                     hands every rank every KV chunk within its d steps: the rank that owns q_chunk
+                     computes such a pair at the step at which the owner of kv_chunk visits.
+    """
+    row_limit, first_query, span_pairs = [], [], []
+    t0 = 0
+    for b, (L, d) in enumerate(zip(seqlens, cp_degrees)):
+        L, d = int(L), int(d)
+        lim = [t0 + i + 1 for i in range(L)]
+        fq = [t0 + i for i in range(L)]
+        for (a, e) in spans_per_seq[b]:
+            for i in range(a, e):
+                lim[i] = t0 + e
+                fq[i] = t0 + a
+        row_limit.extend(lim)
+        first_query.extend(fq)
+        bounds = chunk_bounds(L, d)
+        owner = lambda c: c if c < d else 2 * d - 1 - c
+        for qc in range(2 * d):
+            for kc in range(qc + 1, 2 * d):
+                # some row of q_chunk sees some key of kv_chunk: a span reaches from one into the other
+                if any(max(a, bounds[qc]) < min(e, bounds[qc + 1]) and max(a, bounds[kc]) < min(e, bounds[kc + 1])
+                       for (a, e) in spans_per_seq[b]):
+                    r = owner(qc)
+                    span_pairs.append((b, r, (r - owner(kc)) % d, qc, kc))
+        t0 += L
+    span_pairs.sort()
+    return dict(row_limit=row_limit, first_query=first_query, span_pairs=span_pairs)
+
+
 # ---------------------------------------------------------------------------------------------
 # strategy planner
 # ---------------------------------------------------------------------------------------------

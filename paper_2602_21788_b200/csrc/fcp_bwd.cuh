@@ -157,7 +157,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
   volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
   volatile int* work_ring = (volatile int*)(smem + SM::MISC_OFF + 8);    // [2 slots][unit, kv head]
-  const WaitCtx wctx{abort_flag, a.status};
+  const WaitCtx wctx{abort_flag, a.status, (uint32_t)FCP_WAIT_NS};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 

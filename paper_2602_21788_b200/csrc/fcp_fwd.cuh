@@ -78,7 +78,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             B_TURN = B_SFULL + 8, B_STATFULL = B_SFULL + 10, B_STATEMPTY = B_SFULL + 12;
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
   volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
-  const WaitCtx wctx{abort_flag, a.status};
+  const WaitCtx wctx{abort_flag, a.status, (uint32_t)FCP_WAIT_NS};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 

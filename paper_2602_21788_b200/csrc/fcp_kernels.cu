@@ -876,3 +876,44 @@ extern "C" int fcp_noalloc_device_status(int32_t* status) {
   FCP_CUDA_CHECK(cudaMemcpy(status, g_noalloc_ptr[dev], 4 * sizeof(int32_t), cudaMemcpyDeviceToHost));
   return FCP_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Self-test of the bounded device-side wait
+// ---------------------------------------------------------------------------------------------
+// One CTA of one warp; lane 0 waits, through the same mbar_wait / wait_teardown the persistent kernels
+// use, on a barrier that nobody will ever arrive at.  The wait limit is an argument (a millisecond or
+// so instead of the kernels' two seconds), so the launch ends by itself after about that long.  The
+// status words are a device array of their own: no plan is involved and none is marked as failed.
+static __device__ int32_t g_wait_probe_status[4];
+
+__global__ void __launch_bounds__(32) fcp_wait_probe_kernel(uint32_t limit_ns, int where) {
+  __shared__ __align__(8) unsigned long long bar;
+  __shared__ int abort_flag;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    mbar_init(b, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  const WaitCtx ctx{&abort_flag, g_wait_probe_status, limit_ns};
+  if (threadIdx.x == 0) (void)mbar_wait(b, 0, ctx, where);     // phase 0 never completes
+  __syncwarp();
+  wait_teardown(ctx);
+}
+
+extern "C" int fcp_selftest_bounded_wait(uint32_t limit_us, int32_t* status, void* stream) {
+  if (!status || limit_us == 0 || limit_us > 100000u) {
+    fcp_set_error("fcp_selftest_bounded_wait: status is NULL or the limit is outside [1, 100000] microseconds");
+    return FCP_ERR_INVALID_ARG;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  void* dst = nullptr;
+  FCP_CUDA_CHECK(cudaGetSymbolAddress(&dst, g_wait_probe_status));
+  FCP_CUDA_CHECK(cudaMemsetAsync(dst, 0, 4 * sizeof(int32_t), st));
+  fcp_wait_probe_kernel<<<1, 32, 0, st>>>(limit_us * 1000u, 901);
+  FCP_CUDA_CHECK(cudaGetLastError());
+  FCP_CUDA_CHECK(cudaMemcpyAsync(status, dst, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  FCP_CUDA_CHECK(cudaStreamSynchronize(st));
+  return FCP_OK;
+}

@@ -78,6 +78,7 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
 struct WaitCtx {
   volatile int* abort_flag;
   int* status;                // global: [0] status, [1] where, [2] block, [3] reserved
+  uint32_t limit_ns;          // a wait gives up after this long without progress (below 2^32 ns)
 };
 
 // Bounded wait.  Returns false if the CTA is aborting (this waiter timed out, or another did).
@@ -97,7 +98,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const W
       const uint32_t now = globaltimer_lo();
       if (spins == 2048u) t0 = now;
       const int flag = *ctx.abort_flag;
-      if (flag != 0 || now - t0 > (uint32_t)FCP_WAIT_NS) {
+      if (flag != 0 || now - t0 > ctx.limit_ns) {
         if (flag == 0) *ctx.abort_flag = 0x40000000 | where;
         return false;
       }

@@ -29,7 +29,7 @@ EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_inf
            "fcp_attn_fwd_fused", "fcp_lse_merge", "fcp_attn_bwd", "fcp_attn_bwd_heads",
            "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
            "fcp_plan_kernel_ms", "fcp_noalloc_bytes_needed", "fcp_attn_bwd_noalloc", "fcp_noalloc_device_status",
-           "fcp_status_string",
+           "fcp_selftest_bounded_wait", "fcp_status_string",
            "fcp_last_error_message"]
 
 
@@ -84,6 +84,7 @@ def lib() -> C.CDLL:
     L.fcp_noalloc_bytes_needed.argtypes = [vp, i64p]
     L.fcp_attn_bwd_noalloc.argtypes = [vp] * 11
     L.fcp_noalloc_device_status.argtypes = [i32p]
+    L.fcp_selftest_bounded_wait.argtypes = [C.c_uint32, i32p, vp]
     L.fcp_status_string.argtypes = [C.c_int]
     L.fcp_status_string.restype = C.c_char_p
     L.fcp_last_error_message.restype = C.c_char_p
@@ -266,4 +267,12 @@ def fcp_attn_bwd_noalloc(plan: Plan, q, k, v, o, d_o, lse, dq, dk, dv, stream=0)
 def fcp_noalloc_device_status():
     st = np.zeros(4, dtype=np.int32)
     _check(lib().fcp_noalloc_device_status(st.ctypes.data_as(C.POINTER(C.c_int32))))
+    return st
+
+
+def fcp_selftest_bounded_wait(limit_us=1000, stream=0):
+    """Makes one bounded device-side wait run out on purpose (a barrier nobody arrives at, limit in
+    microseconds) and returns the four status words it produced."""
+    st = np.zeros(4, dtype=np.int32)
+    _check(lib().fcp_selftest_bounded_wait(int(limit_us), st.ctypes.data_as(C.POINTER(C.c_int32)), C.c_void_p(stream)))
     return st

@@ -92,6 +92,18 @@ class Workload:
     def flops_fwd_bwd(self) -> float:
         return 3.5 * self.flops_fwd()
 
+    def device_tensors(self, with_do: bool = True):
+        """The same distributions drawn on the current CUDA device by torch's seeded generator, as bf16
+        tensors: for workloads whose host draw would take minutes (billions of values).  A pure
+        function of (seed, shape) like `tensors`, but a different stream of numbers."""
+        import torch
+        g = torch.Generator(device="cuda")
+        g.manual_seed(0xFC9 + 7919 * int(self.seed))
+        T, D = self.total_tokens, self.head_dim
+        mk = lambda h: torch.randn((T, h, D), dtype=torch.bfloat16, device="cuda", generator=g)
+        out = (mk(self.hq), mk(self.hkv), mk(self.hkv))
+        return out + (mk(self.hq),) if with_do else out
+
     def tensors(self, with_do: bool = True):
         """q[T,hq,D], k[T,hkv,D], v[T,hkv,D] (and dO[T,hq,D]) as bf16 bit patterns (uint16)."""
         rng = np.random.Generator(np.random.PCG64([self.seed, 0xFC9]))

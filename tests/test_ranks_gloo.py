@@ -58,3 +58,25 @@ def test_single_process_is_the_identity():
     assert ranks.aggregate(3.5, 7.0, "cpu") == (3.5, 7.0)
     w = ranks.rank_workload("tiny", seed=2, rank=0, world=1)
     assert w.seqlens.tolist() == synth.make_workload("tiny", seed=2).seqlens.tolist()
+
+
+def test_bench_gpus_n_starts_its_own_ranks():
+    """`python bench.py --gpus 2` run plainly (no WORLD_SIZE in the environment) starts two ranks through
+    torch.distributed.run and rank 0 prints one JSON line with n_gpus = 2.  Here on CPU: `gloo` ranks and a
+    sleep in place of the GPU step (`--selftest-launcher`), the same rank plumbing as the measured path."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--steps", "2", "--selftest-launcher"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    out = json.loads(lines[0])
+    assert out["n_gpus"] == 2 and out["selftest"] == "launcher" and out["value"] is None
+    f0 = synth.make_workload("tiny", 0).flops_fwd_bwd()
+    f1 = synth.make_workload("tiny", 1).flops_fwd_bwd()
+    assert out["flops_rank0"] == f0 and out["flops_all_ranks"] == f0 + f1      # seed = rank: different batches, summed
+    assert out["max_ms_over_ranks"] >= 20.0                                    # rank 1 sleeps 20 ms: max over ranks

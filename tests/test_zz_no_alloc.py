@@ -4,7 +4,8 @@ Some users of the library reach the backward pass in a place where they may not 
 memory: every byte belongs to their framework's pool, cudaMalloc would stall or is off limits
 there, or the device is simply full.  fcp_attn_bwd_noalloc serves them from an array built into the
 library, needs no uploaded plan and no scratch argument.  It has to give the same gradients as
-fcp_attn_bwd on the same inputs, also when it is called twice in a row (the built-in array keeps
+fcp_attn_bwd on the same inputs (and, like it, the fp64 oracle's within the parity tolerance), also
+when it is called twice in a row (the built-in array keeps
 the first call's contents, so the second call checks that everything that must be cleared is).
 
 Collected last on purpose: with `-x` every other test has run before this one can fail.
@@ -12,6 +13,7 @@ Collected last on purpose: with `-x` every other test has run before this one ca
 import numpy as np
 import pytest
 
+from oracle import attention_ref as A
 from paper_2602_21788_b200 import build, synth
 
 pytestmark = pytest.mark.gpu
@@ -43,6 +45,8 @@ def test_noalloc_backward_matches_regular_backward_twice(lens, degs, hq, hkv, D)
     torch.cuda.synchronize()
     ds.check_status()
     ref = {n: synth.bf16_bits_to_f64(_bits(getattr(ds, n))) for n in ("dq", "dk", "dv")}
+    f = synth.bf16_bits_to_f64
+    oracle = dict(zip(("dq", "dk", "dv"), A.attention_bwd_packed(f(q), f(k), f(v), f(do), w.cu_seqlens)))
 
     host_plan = fcp.fcp_plan_blocks(w.seqlens, w.cp_degrees, hq, hkv, D)       # never uploaded
     assert fcp.fcp_noalloc_bytes_needed(host_plan) <= fcp.FCP_NOALLOC_MAX_BYTES
@@ -60,6 +64,9 @@ def test_noalloc_backward_matches_regular_backward_twice(lens, degs, hq, hkv, D)
         g = synth.bf16_bits_to_f64(_bits(got["dq"]))  # fp32 reductions in varying order: the tests' tolerance
         assert np.isfinite(g).all()
         assert np.linalg.norm(g - ref["dq"]) <= 2e-2 * np.linalg.norm(ref["dq"]), call
+        for n in ("dq", "dk", "dv"):                 # and the fp64 oracle's gradients, at the parity tests' tolerance
+            x = synth.bf16_bits_to_f64(_bits(got[n]))
+            assert np.linalg.norm(x - oracle[n]) <= 2e-2 * np.linalg.norm(oracle[n]), (n, call)
 
 
 def test_noalloc_rejects_batches_beyond_the_builtin_arena():
