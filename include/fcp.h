@@ -98,6 +98,28 @@ int fcp_plan_strategy(const int32_t* seqlens, int32_t B, int32_t N, double E, do
 int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
                     const fcp_params* params, fcp_plan** plan);
 
+/* ------------------------------------------------------------------------------------------
+ * fcp_plan_blocks_spans — host only.  fcp_plan_blocks for sequences that carry bidirectional spans:
+ * multimodal batches let the tokens of an image or a video frame attend to each other in both
+ * directions while text stays causal, which is what the mask efficiency factor eta_k > 0 of the
+ * cost model stands for (Sec. 4.3, Eq. 4).  Sequence b has the spans span_offset[b] ..
+ * span_offset[b+1]-1 of `spans`, each a pair (begin, end) of positions relative to the sequence
+ * start, sorted, disjoint, 0 <= begin < end <= length.  Query i sees key j iff j <= i, or both lie
+ * in the same span; so query t sees exactly the keys before FCP_TABLE_ROW_LIMIT[t] and key t is
+ * seen from query FCP_TABLE_FIRST_QUERY[t] on.  The causal tables (pairs, items, slots) are those
+ * of fcp_plan_blocks; FCP_TABLE_SPAN_PAIRS lists the block pairs above the chunk diagonal that the
+ * spans add (computed by the rank that owns the Q chunk when the KV chunk's owner visits).
+ * fcp_attn_fwd_fused and fcp_attn_bwd apply the mask; the per-item partial path (fcp_attn_fwd,
+ * fcp_attn_fwd_merged, fcp_lse_merge) and fcp_attn_bwd_noalloc are causal only and return
+ * FCP_ERR_UNSUPPORTED for such a plan.  span_offset == NULL means no spans.
+ * fcp_span_mask_efficiency gives the eta_k of one sequence for fcp_plan_strategy: visible
+ * (query, key) pairs over the causal count L(L+1)/2, minus 1.
+ */
+int fcp_plan_blocks_spans(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
+                          const int32_t* span_offset, const int32_t* spans,
+                          const fcp_params* params, fcp_plan** plan);
+int fcp_span_mask_efficiency(int32_t length, const int32_t* spans, int32_t n_spans, double* eta);
+
 /* Tables readable through fcp_plan_get.  All are int32, row-major, host memory owned by the plan.
  * Rows are in the canonical order (sequence, rank, step, q_chunk, kv_chunk).                     */
 #define FCP_TABLE_CU_SEQLENS    0  /* [B+1]                     packed-token offsets of the sequences */
@@ -113,6 +135,9 @@ int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B
 #define FCP_TABLE_MERGE_UNITS  10  /* [n_merge_units][4]        derived                               */
 #define FCP_TABLE_BWD_WORK     11  /* [n_bwd_units]             derived: backward units in execution order (per KV head) */
 #define FCP_TABLE_FUSED_UNITS  12  /* [n_fused_units][16]       derived: work units of fcp_attn_fwd_fused       */
+#define FCP_TABLE_ROW_LIMIT    13  /* [T] or empty              first key (packed index) query t does not see   */
+#define FCP_TABLE_FIRST_QUERY  14  /* [T] or empty              first query (packed index) that sees key t      */
+#define FCP_TABLE_SPAN_PAIRS   15  /* [n][5]  seq, rank, step, q_chunk, kv_chunk (> q_chunk): pairs a span adds  */
 
 /* fcp_plan_get: *host_ptr = first element of the table, *count = number of int32 elements. */
 int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count);

@@ -65,6 +65,7 @@ struct BwdArgs {
   float scale, scale_log2;
   const float* delta_t;     // [hq_acc][t_stride], already multiplied by the softmax scale
   const float* lse2_t;      // [hq_acc][t_stride], log2 units
+  const int32_t* first_query;   // [T] or nullptr (causal): first query (packed index) that sees key t
   float* dq_acc;            // [T][hq_acc][D] fp32, zero-initialised
   __nv_bfloat16* dk;        // [T][hkv][D]
   __nv_bfloat16* dv;
@@ -77,7 +78,7 @@ struct BwdArgs {
 // share) to one head's worth of L2.
 struct BwdIter {
   const int32_t* qr;     // Q ranges of the unit
-  int nq, kv_tile, g;
+  int nq, t_first, t_mask_end, g;   // a DIAG range starts at Q tile t_first; tiles before t_mask_end need the mask
   int r, t, hh;          // range, tile within range, head within group
   int qb, qe, diag;
   bool valid;
@@ -89,7 +90,7 @@ struct BwdIter {
     qb = __ldg(Q + BQ_BEGIN);
     qe = __ldg(Q + BQ_END);
     diag = __ldg(Q + BQ_DIAG);
-    t = diag ? kv_tile : 0;
+    t = diag ? t_first : 0;
   }
   __device__ __forceinline__ void settle() {           // make (hh, r, t) point at an existing tile
     while (valid && qb + t * 128 >= qe) {
@@ -102,13 +103,14 @@ struct BwdIter {
     if (valid) {
       q_row = qb + t * 128;
       q_valid = min(128, qe - q_row);
-      causal = diag && t == kv_tile;
+      causal = diag && t < t_mask_end;
     }
   }
   __device__ __forceinline__ void init(const int32_t* U, const int32_t* qranges, int g_) {
     qr = qranges + (size_t)__ldg(U + BU_FIRST_QRANGE) * FCP_BWD_QRANGE_W;
     nq = __ldg(U + BU_N_QRANGES);
-    kv_tile = __ldg(U + BU_KV_TILE);
+    t_first = __ldg(U + BU_T_FIRST);
+    t_mask_end = __ldg(U + BU_T_MASK_END);
     g = g_;
     r = 0; hh = 0;
     valid = nq > 0;
@@ -356,6 +358,8 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int32_t* U = next_work(n++, hk, ok);
       if (!U) break;
       const int kv_row0 = __ldg(U + BU_KV_ROW0), kv_rows = __ldg(U + BU_KV_ROWS);
+      // first query that sees this thread's key row: the key itself, or the begin of its span
+      const int first_q = (a.first_query != nullptr && row < kv_rows) ? __ldg(a.first_query + kv_row0 + row) : kv_row0 + row;
       BwdIter iter;
       iter.init(U, a.qranges, g);
       float pre = load_row(iter, hk);
@@ -391,7 +395,7 @@ fcp_bwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           // valid query columns of this key row, relative to this warp's half: [lo, hi).  Bit j of
           // `keep` = column j survives; applied to the packed pairs.
           const int hi = min(64, max(0, (row < kv_rows ? q_valid : 0) - half * 64));
-          const int lo = min(64, max(0, (causal ? kv_row0 + row - q_row : 0) - half * 64));
+          const int lo = min(64, max(0, (causal ? first_q - q_row : 0) - half * 64));
           keep = (hi > lo) ? ((hi == 64 ? ~0ull : ((1ull << hi) - 1)) & ~((1ull << lo) - 1)) : 0ull;
         }
 #pragma unroll 1

@@ -55,6 +55,7 @@ struct FwdArgs {
   __nv_bfloat16* o_direct;   // [T][hq][D] or nullptr: final output of Q chunks that have a single slot
   float* lse_direct;         // [T][hq]
   float* o_f32_direct;       // [T][hq][D] or nullptr: the rows written to o_direct before their rounding to bf16
+  const int32_t* row_limit;  // [T] or nullptr (causal): first key (packed index) that query t does not see
   int32_t* status;        // [4]
 };
 
@@ -264,6 +265,8 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int nts = __ldg(U + FU_NT_STAGE0 + s);
       const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
       const int q_pos = __ldg(U + FU_Q_ROW0) + s * 128 + row;
+      // first key this row does not see in a DIAG range: the one after itself, or the end of its span
+      const int row_lim = (a.row_limit != nullptr && s * 128 + row < __ldg(U + FU_Q_ROWS)) ? __ldg(a.row_limit + q_pos) : q_pos + 1;
       const int nr0 = __ldg(U + FU_NT_RANGE0);
       const int kvb0 = __ldg(U + FU_KV0_BEGIN), kvb1 = __ldg(U + FU_KV1_BEGIN);
       const int kve0 = __ldg(U + FU_KV0_END), kve1 = __ldg(U + FU_KV1_END);
@@ -285,7 +288,7 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const bool r1 = j >= nr0;
         const int ks = r1 ? kvb1 + (j - nr0) * 128 : kvb0 + j * 128;
         int limit = (r1 ? kve1 : kve0) - ks;                  // valid columns of this tile for this row
-        if (r1 ? kvd1 : kvd0) limit = min(limit, q_pos - ks + 1);
+        if (r1 ? kvd1 : kvd0) limit = min(limit, row_lim - ks);
         const bool masked = __any_sync(0xffffffffu, limit < 128);
         ok = mbar_wait_warp(BAR(B_SFULL + s), scnt & 1, wctx, 30 + s);
         ++scnt;

@@ -218,9 +218,10 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   }
   plan->device = dev;
   plan->sm_count = prop.multiProcessorCount;
-  constexpr int NT = 8;
+  constexpr int NT = 10;
   const std::vector<int32_t>* tabs[NT] = {&plan->fwd_units, &plan->bwd_units, &plan->bwd_qranges, &plan->merge_units,
-                                          &plan->slot_offset, &plan->slot_rows, &plan->bwd_work, &plan->fused_units};
+                                          &plan->slot_offset, &plan->slot_rows, &plan->bwd_work, &plan->fused_units,
+                                          &plan->row_limit, &plan->first_query};
   size_t off[NT + 1];
   size_t total = 256;  // status words first
   for (int i = 0; i < NT; ++i) {
@@ -251,6 +252,8 @@ extern "C" int fcp_plan_upload(fcp_plan* plan, void* stream) {
   plan->d_slot_rows = (int32_t*)((char*)blob + off[5]);
   plan->d_bwd_work = (int32_t*)((char*)blob + off[6]);
   plan->d_fused_units = (int32_t*)((char*)blob + off[7]);
+  plan->d_row_limit = plan->row_limit.empty() ? nullptr : (int32_t*)((char*)blob + off[8]);
+  plan->d_first_query = plan->first_query.empty() ? nullptr : (int32_t*)((char*)blob + off[9]);
   // opt in to the large dynamic shared memory of the tensor-core kernels once
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<64>::DYN_BYTES));
   FCP_CUDA_CHECK(cudaFuncSetAttribute(fcp_fwd_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdSmem<128>::DYN_BYTES));
@@ -362,6 +365,11 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
     return FCP_ERR_INVALID_ARG;
   }
   if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+  if (!fused && !plan->row_limit.empty()) {
+    fcp_set_error("the per-item partial path (fcp_attn_fwd, fcp_attn_fwd_merged) is causal only; a plan with "
+                  "bidirectional spans runs through fcp_attn_fwd_fused");
+    return FCP_ERR_UNSUPPORTED;
+  }
   const fcp_params& P = plan->params;
   CUtensorMap tq, tk, tv;
   if ((rc = make_thd_map(&tq, q, plan->T, P.hq, P.head_dim, 128)) != FCP_OK) return rc;
@@ -384,6 +392,7 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
   a.o_direct = (__nv_bfloat16*)o_direct;
   a.lse_direct = lse_direct;
   a.o_f32_direct = o_f32_direct;
+  a.row_limit = fused ? plan->d_row_limit : nullptr;
   a.status = plan->d_status;
   const int64_t n_work = (int64_t)a.n_units * head_count;
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
@@ -447,6 +456,10 @@ extern "C" int fcp_lse_merge(const fcp_plan* plan, const float* o_partial, const
     return FCP_ERR_INVALID_ARG;
   }
   if ((rc = check_heads(plan, head_begin, head_count)) != FCP_OK) return rc;
+  if (!plan->row_limit.empty()) {
+    fcp_set_error("fcp_lse_merge: the per-item partial path is causal only; this plan has bidirectional spans");
+    return FCP_ERR_UNSUPPORTED;
+  }
   return launch_merge(plan, o_partial, lse_partial, head_begin, head_count, o, o_f32, lse,
                       (int)(plan->merge_units.size() / FCP_MERGE_UNIT_W), stream);
 }
@@ -456,7 +469,7 @@ namespace {
 // work counter, SM count.  fcp_attn_bwd_heads takes them from the uploaded plan, fcp_attn_bwd_noalloc
 // from the built-in arena.
 struct BwdTables {
-  const int32_t *units, *qranges, *order;
+  const int32_t *units, *qranges, *order, *first_query;
   int32_t* status;
   int32_t* counter;
   int sm_count;
@@ -519,6 +532,7 @@ int run_bwd(const fcp_plan* plan, const BwdTables& tb, const void* q, const void
   a.delta_t = delta_t;
   a.lse2_t = lse2_t;
   a.dq_acc = dq_acc;
+  a.first_query = tb.first_query;
   a.dk = (__nv_bfloat16*)dk;
   a.dv = (__nv_bfloat16*)dv;
   a.status = tb.status;
@@ -569,8 +583,8 @@ extern "C" int fcp_attn_bwd_heads(const fcp_plan* plan, const void* q, const voi
     fcp_set_error("fcp_attn_bwd: scratch of %lld bytes, %lld needed", (long long)scratch_bytes, (long long)need);
     return FCP_ERR_WORKSPACE;
   }
-  const BwdTables tb{plan->d_bwd_units, plan->d_bwd_qranges, plan->d_bwd_work, plan->d_status, plan->d_status + 16,
-                     plan->sm_count};
+  const BwdTables tb{plan->d_bwd_units, plan->d_bwd_qranges, plan->d_bwd_work, plan->d_first_query, plan->d_status,
+                     plan->d_status + 16, plan->sm_count};
   return run_bwd(plan, tb, q, k, v, o, d_o, lse, kv_head_begin, kv_head_count, dq, dk, dv, scratch, plan,
                  (cudaStream_t)stream);
 }
@@ -653,7 +667,15 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
       while (b1 < B - (want - 1 - g) && plan->cu_seqlens[b1] < target) ++b1;
     }
     fcp_plan* sub = nullptr;
-    int rc = fcp_plan_blocks(lens.data() + b0, degs.data() + b0, b1 - b0, &plan->params, &sub);
+    int rc;
+    if (plan->span_offset.empty()) {
+      rc = fcp_plan_blocks(lens.data() + b0, degs.data() + b0, b1 - b0, &plan->params, &sub);
+    } else {                                     // the run's spans, offsets counted from its first one
+      std::vector<int32_t> so(b1 - b0 + 1);
+      for (int b = b0; b <= b1; ++b) so[b - b0] = plan->span_offset[b] - plan->span_offset[b0];
+      rc = fcp_plan_blocks_spans(lens.data() + b0, degs.data() + b0, b1 - b0, so.data(),
+                                 plan->spans.data() + 2 * (size_t)plan->span_offset[b0], &plan->params, &sub);
+    }
     if (rc == FCP_OK) rc = fcp_plan_upload(sub, stream);
     if (rc != FCP_OK) {
       if (sub) fcp_plan_destroy(sub);
@@ -822,6 +844,10 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
     fcp_set_error("fcp_attn_bwd_noalloc: NULL argument");
     return FCP_ERR_INVALID_ARG;
   }
+  if (!plan->first_query.empty()) {
+    fcp_set_error("fcp_attn_bwd_noalloc: plans with bidirectional spans are not supported here; use fcp_attn_bwd");
+    return FCP_ERR_UNSUPPORTED;
+  }
   int64_t need = 0;
   fcp_noalloc_bytes_needed(plan, &need);
   if (need > (int64_t)FCP_NOALLOC_MAX_BYTES) {
@@ -860,7 +886,7 @@ extern "C" int fcp_attn_bwd_noalloc(const fcp_plan* plan, const void* q, const v
   if (!plan->bwd_work.empty())
     FCP_CUDA_CHECK(cudaMemcpyAsync(d_work, plan->bwd_work.data(), plan->bwd_work.size() * 4, cudaMemcpyHostToDevice, st));
 
-  const BwdTables tb{d_units, d_qranges, d_work, d_status, d_status + 16, g_noalloc_sms[dev]};
+  const BwdTables tb{d_units, d_qranges, d_work, nullptr, d_status, d_status + 16, g_noalloc_sms[dev]};
   return run_bwd(plan, tb, q, k, v, o, d_o, lse, 0, P.hkv, dq, dk, dv, d_scratch, nullptr, st);
 }
 

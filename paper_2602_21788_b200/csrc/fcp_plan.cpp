@@ -177,7 +177,13 @@ inline int ceil_div(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
 
 extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
                                const fcp_params* params, fcp_plan** out) {
-  if (!seqlens || !cp_degrees || !params || !out || B <= 0) {
+  return fcp_plan_blocks_spans(seqlens, cp_degrees, B, nullptr, nullptr, params, out);
+}
+
+extern "C" int fcp_plan_blocks_spans(const int32_t* seqlens, const int32_t* cp_degrees, int32_t B,
+                                     const int32_t* span_offset, const int32_t* spans,
+                                     const fcp_params* params, fcp_plan** out) {
+  if (!seqlens || !cp_degrees || !params || !out || B <= 0 || (span_offset && !spans && span_offset[B] > 0)) {
     fcp_set_error("fcp_plan_blocks: invalid argument");
     return FCP_ERR_INVALID_ARG;
   }
@@ -212,6 +218,43 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
   p->T = T;
   p->cu_seqlens.assign(B + 1, 0);
   for (int b = 0; b < B; ++b) p->cu_seqlens[b + 1] = p->cu_seqlens[b] + seqlens[b];
+
+  // Bidirectional spans: query t sees the keys before row_limit[t]; key t is seen from query
+  // first_query[t] on (both in packed-token indices, both non-decreasing within a sequence).
+  const bool has_spans = span_offset != nullptr && span_offset[B] > span_offset[0];
+  if (has_spans) {
+    p->span_offset.assign(span_offset, span_offset + B + 1);
+    p->spans.assign(spans, spans + 2 * (size_t)span_offset[B]);
+    p->row_limit.resize(T);
+    p->first_query.resize(T);
+    for (int64_t t = 0; t < T; ++t) {
+      p->row_limit[t] = (int32_t)t + 1;
+      p->first_query[t] = (int32_t)t;
+    }
+    for (int b = 0; b < B; ++b) {
+      int32_t prev_end = 0;
+      if (span_offset[b + 1] < span_offset[b]) {
+        delete p;
+        fcp_set_error("fcp_plan_blocks_spans: span_offset decreases at sequence %d", b);
+        return FCP_ERR_INVALID_ARG;
+      }
+      for (int32_t i = span_offset[b]; i < span_offset[b + 1]; ++i) {
+        const int32_t a = spans[2 * i], e = spans[2 * i + 1];
+        if (a < prev_end || e <= a || e > seqlens[b]) {
+          delete p;
+          fcp_set_error("fcp_plan_blocks_spans: span [%d, %d) of sequence %d (length %d) is empty, out of range, "
+                        "unsorted or overlaps the one before", a, e, b, seqlens[b]);
+          return FCP_ERR_INVALID_ARG;
+        }
+        prev_end = e;
+        const int32_t t0 = p->cu_seqlens[b];
+        for (int32_t t = a; t < e; ++t) {
+          p->row_limit[t0 + t] = t0 + e;
+          p->first_query[t0 + t] = t0 + a;
+        }
+      }
+    }
+  }
 
   // Chunk bounds and pairs.
   p->chunk_offset.push_back(0);
@@ -250,6 +293,34 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
   for (const Pair& x : pairs) {
     const int32_t row[6] = {x.seq, x.rank, x.step, x.qc, x.kc, x.kind};
     p->pairs.insert(p->pairs.end(), row, row + 6);
+  }
+  // Block pairs above the chunk diagonal that a span makes necessary: (q_chunk, kv_chunk > q_chunk) such that
+  // a span reaches into both.  The rank that owns q_chunk computes it when the owner of kv_chunk visits.
+  if (has_spans) {
+    for (int b = 0; b < B; ++b) {
+      const int d = cp_degrees[b];
+      const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
+      const int32_t t0 = cbp[0];
+      std::vector<Pair> sp;
+      auto owner = [&](int c) { return c < d ? c : 2 * d - 1 - c; };
+      for (int qc = 0; qc < 2 * d; ++qc)
+        for (int kc = qc + 1; kc < 2 * d; ++kc) {
+          bool hit = false;
+          for (int32_t i = span_offset[b]; i < span_offset[b + 1] && !hit; ++i) {
+            const int32_t a = t0 + spans[2 * i], e = t0 + spans[2 * i + 1];
+            hit = std::max(a, cbp[qc]) < std::min(e, cbp[qc + 1]) && std::max(a, cbp[kc]) < std::min(e, cbp[kc + 1]);
+          }
+          if (hit) {
+            const int r = owner(qc);
+            sp.push_back(Pair{b, r, ((r - owner(kc)) % d + d) % d, qc, kc, 2});
+          }
+        }
+      std::sort(sp.begin(), sp.end());
+      for (const Pair& x : sp) {
+        const int32_t row[5] = {x.seq, x.rank, x.step, x.qc, x.kc};
+        p->span_pairs.insert(p->span_pairs.end(), row, row + 5);
+      }
+    }
   }
 
   // Items: one per (seq, rank, step, q_chunk); slot = order of the step among the steps touching
@@ -373,17 +444,21 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
   }
   {
     std::vector<FU> gus;
-    auto emit_run = [&](int32_t t0, int32_t r0, int32_t r1) {     // rows [r0, r1) attend to [t0, row]
+    // rows [r0, r1) of the sequence [t0, t1) attend to [t0, row] (and, inside a span, on to the span's end)
+    auto emit_run = [&](int32_t t0, int32_t t1, int32_t r0, int32_t r1) {
       for (int32_t off = 0; off < r1 - r0; off += FCP_FWD_UNIT_ROWS) {
         FU u{};
         const int32_t rows = std::min<int32_t>(FCP_FWD_UNIT_ROWS, r1 - r0 - off);
         u.f[FU_Q_ROW0] = r0 + off;
         u.f[FU_Q_ROWS] = rows;
         u.f[FU_N_RANGES] = 1;
-        u.f[FU_KV0_BEGIN] = t0; u.f[FU_KV0_END] = r1; u.f[FU_KV0_DIAG] = 1;
+        u.f[FU_KV0_BEGIN] = t0; u.f[FU_KV0_END] = has_spans ? t1 : r1; u.f[FU_KV0_DIAG] = 1;
         for (int s = 0; s < 2; ++s) {
           const int32_t rs = std::min<int32_t>(FCP_TILE, rows - s * FCP_TILE);
-          u.f[FU_NT_STAGE0 + s] = rs > 0 ? ceil_div((int64_t)(r0 + off - t0) + s * FCP_TILE + rs, FCP_TILE) : 0;
+          // key tiles up to the last key the stage's last row sees (row limits do not decrease along a sequence)
+          const int32_t last_row = r0 + off + s * FCP_TILE + rs - 1;
+          const int32_t key_end = rs > 0 ? (has_spans ? p->row_limit[last_row] : last_row + 1) : t0;
+          u.f[FU_NT_STAGE0 + s] = rs > 0 ? ceil_div(key_end - t0, FCP_TILE) : 0;
         }
         u.f[FU_NT_RANGE0] = 0x7fffffff;
         u.f[FU_ITEM] = -1;
@@ -393,7 +468,7 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
     };
     for (int b = 0; b < B; ++b) {
       const int32_t* cbp = &p->chunk_bounds[p->chunk_offset[b]];
-      const int32_t t0 = cbp[0];
+      const int32_t t0 = cbp[0], t1 = cbp[2 * cp_degrees[b]];
       int32_t run0 = -1, run1 = -1;
       for (int c = 0; c < 2 * cp_degrees[b]; ++c) {
         const int32_t q0 = cbp[c], q1 = cbp[c + 1];
@@ -403,13 +478,13 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
                             (rg.size() == 2 && !rg[0].diag && rg[0].b == t0 && rg[0].e == q0 && rg[1].diag && rg[1].b == q0);
         if (prefix) {
           if (run0 < 0) run0 = q0;
-          else if (run1 != q0) { emit_run(t0, run0, run1); run0 = q0; }
+          else if (run1 != q0) { emit_run(t0, t1, run0, run1); run0 = q0; }
           run1 = q1;
           continue;
         }
-        if (run0 >= 0) { emit_run(t0, run0, run1); run0 = -1; }
+        if (run0 >= 0) { emit_run(t0, t1, run0, run1); run0 = -1; }
         // a chunk whose ranges are not a causal prefix keeps them as they are (at most two per unit)
-        if (rg.empty() || rg.size() > 2) {
+        if (rg.empty() || rg.size() > 2 || has_spans) {
           delete p;
           fcp_set_error("fcp_plan_blocks: Q chunk %d of sequence %d has %d disjoint KV ranges", c, b, (int)rg.size());
           return FCP_ERR_UNSUPPORTED;
@@ -438,7 +513,7 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
           gus.push_back(u);
         }
       }
-      if (run0 >= 0) emit_run(t0, run0, run1);
+      if (run0 >= 0) emit_run(t0, t1, run0, run1);
     }
     std::stable_sort(gus.begin(), gus.end(), [](const FU& a, const FU& b) {
       return a.f[FU_NT_STAGE0] + a.f[FU_NT_STAGE1] > b.f[FU_NT_STAGE0] + b.f[FU_NT_STAGE1];
@@ -478,18 +553,29 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
         if (cbp[c + 1] > cbp[c])
           causal_seq = causal_seq && out_r.size() == 1 && out_r[0].diag && out_r[0].b == cbp[c] && out_r[0].e == t1;
       }
-      auto emit_tiles = [&](int32_t k0, int32_t k1, int32_t first, const std::vector<Range>& rg) {
+      // `spans`: the tiles are cut from the sequence start and a DIAG range starts where the first key of the
+      // tile is first seen (earlier than the tile's own position when that key lies inside a span)
+      auto emit_tiles = [&](int32_t k0, int32_t k1, int32_t first, const std::vector<Range>& rg, bool spans_on) {
         for (int32_t off = 0, t = 0; off < k1 - k0; off += FCP_TILE, ++t) {
           BU u{};
+          const int32_t rows = std::min<int32_t>(FCP_TILE, k1 - k0 - off);
           u.f[BU_KV_ROW0] = k0 + off;
-          u.f[BU_KV_ROWS] = std::min<int32_t>(FCP_TILE, k1 - k0 - off);
+          u.f[BU_KV_ROWS] = rows;
           u.f[BU_FIRST_QRANGE] = first;
           u.f[BU_N_QRANGES] = (int32_t)rg.size();
-          u.f[BU_KV_TILE] = t;
+          // Q tiles of a DIAG range run from T_FIRST on; those before T_MASK_END hold (query, key) pairs the
+          // mask removes.  Causal: the tile on the diagonal only.
+          int32_t t_first = t, t_mask_end = t + 1;
+          if (spans_on) {
+            t_first = (p->first_query[k0 + off] - k0) / FCP_TILE;
+            t_mask_end = ceil_div(p->first_query[k0 + off + rows - 1] - k0, FCP_TILE);
+          }
+          u.f[BU_T_FIRST] = t_first;
+          u.f[BU_T_MASK_END] = t_mask_end;
           int cost = 0;
           for (const Range& r : rg) {
             const int nt = ceil_div(r.e - r.b, FCP_TILE);
-            cost += r.diag ? std::max(0, nt - t) : nt;
+            cost += r.diag ? std::max(0, nt - t_first) : nt;
           }
           u.f[BU_COST] = cost;
           u.f[BU_SEQ] = b;
@@ -506,10 +592,15 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
       };
       if (causal_seq) {
         const std::vector<Range> whole{Range{t0, t1, 1}};
-        emit_tiles(t0, t1, push_ranges(whole), whole);
+        emit_tiles(t0, t1, push_ranges(whole), whole, has_spans);
       } else {
+        if (has_spans) {
+          delete p;
+          fcp_set_error("fcp_plan_blocks_spans: sequence %d has spans but its block pairs are not the causal set", b);
+          return FCP_ERR_UNSUPPORTED;
+        }
         for (int c = 0; c < nc; ++c)
-          if (!kv_cover[c].empty()) emit_tiles(cbp[c], cbp[c + 1], push_ranges(kv_cover[c]), kv_cover[c]);
+          if (!kv_cover[c].empty()) emit_tiles(cbp[c], cbp[c + 1], push_ranges(kv_cover[c]), kv_cover[c], false);
       }
     }
   }
@@ -551,6 +642,28 @@ extern "C" int fcp_plan_blocks(const int32_t* seqlens, const int32_t* cp_degrees
   return FCP_OK;
 }
 
+extern "C" int fcp_span_mask_efficiency(int32_t length, const int32_t* spans, int32_t n_spans, double* eta) {
+  if (length <= 0 || !eta || n_spans < 0 || (n_spans > 0 && !spans)) {
+    fcp_set_error("fcp_span_mask_efficiency: invalid argument");
+    return FCP_ERR_INVALID_ARG;
+  }
+  // a span of m tokens adds the m(m-1)/2 pairs above its diagonal to the L(L+1)/2 causal ones
+  double extra = 0.0;
+  int32_t prev_end = 0;
+  for (int i = 0; i < n_spans; ++i) {
+    const int32_t a = spans[2 * i], e = spans[2 * i + 1];
+    if (a < prev_end || e <= a || e > length) {
+      fcp_set_error("fcp_span_mask_efficiency: span [%d, %d) is empty, out of range, unsorted or overlapping", a, e);
+      return FCP_ERR_INVALID_ARG;
+    }
+    prev_end = e;
+    const double m = double(e - a);
+    extra += m * (m - 1.0) / 2.0;
+  }
+  *eta = extra / (double(length) * (double(length) + 1.0) / 2.0);
+  return FCP_OK;
+}
+
 extern "C" int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t** host_ptr, int64_t* count) {
   if (!plan || !host_ptr || !count) return FCP_ERR_INVALID_ARG;
   const std::vector<int32_t>* v = nullptr;
@@ -568,6 +681,9 @@ extern "C" int fcp_plan_get(const fcp_plan* plan, int32_t which, const int32_t**
     case FCP_TABLE_MERGE_UNITS: v = &plan->merge_units; break;
     case FCP_TABLE_BWD_WORK: v = &plan->bwd_work; break;
     case FCP_TABLE_FUSED_UNITS: v = &plan->fused_units; break;
+    case FCP_TABLE_ROW_LIMIT: v = &plan->row_limit; break;
+    case FCP_TABLE_FIRST_QUERY: v = &plan->first_query; break;
+    case FCP_TABLE_SPAN_PAIRS: v = &plan->span_pairs; break;
     default: fcp_set_error("fcp_plan_get: unknown table %d", which); return FCP_ERR_INVALID_ARG;
   }
   *host_ptr = v->data();

@@ -20,7 +20,7 @@ enum {
   FU_NT_STAGE0, FU_NT_STAGE1, FU_NT_RANGE0, FU_ITEM, FU_SINGLE_SLOT, FU_RSV1
 };
 // Field indices of a backward unit row and of a Q range row.
-enum { BU_KV_ROW0 = 0, BU_KV_ROWS, BU_FIRST_QRANGE, BU_N_QRANGES, BU_KV_TILE, BU_COST, BU_SEQ, BU_RSV };
+enum { BU_KV_ROW0 = 0, BU_KV_ROWS, BU_FIRST_QRANGE, BU_N_QRANGES, BU_T_FIRST, BU_COST, BU_SEQ, BU_T_MASK_END };
 enum { BQ_BEGIN = 0, BQ_END, BQ_DIAG, BQ_RSV };
 enum { MU_TOK_BEGIN = 0, MU_N_TOK, MU_CHUNK, MU_CHUNK_TOK_BEGIN };
 
@@ -32,6 +32,8 @@ struct fcp_plan {
   int32_t n_merge_multi = 0;   // merge units of chunks with two or more slots (they come first in merge_units)
   std::vector<int32_t> cu_seqlens, chunk_offset, chunk_bounds, pairs, items, slot_offset, slot_rows;
   std::vector<int32_t> fwd_units, bwd_units, bwd_qranges, merge_units, bwd_work, fused_units;
+  std::vector<int32_t> row_limit, first_query, span_pairs;   // empty unless the plan has bidirectional spans
+  std::vector<int32_t> span_offset, spans;                   // the caller's span list ([B+1], [n][2]); empty if none
 
   // device copy (fcp_plan_upload)
   int device = -1;
@@ -42,6 +44,8 @@ struct fcp_plan {
   int32_t* d_merge_units = nullptr;
   int32_t* d_bwd_work = nullptr;
   int32_t* d_fused_units = nullptr;
+  int32_t* d_row_limit = nullptr;      // nullptr for a causal plan
+  int32_t* d_first_query = nullptr;
   int32_t* d_slot_offset = nullptr;
   int32_t* d_slot_rows = nullptr;
   int32_t* d_status = nullptr; // [4]: status word, diagnostic

@@ -19,12 +19,14 @@ FCP_ERR_CUDA, FCP_ERR_TIMEOUT, FCP_ERR_NOT_UPLOADED = -5, -6, -7
 FCP_MAX_DEGREE = 64
 
 TABLES = dict(cu_seqlens=0, chunk_offset=1, chunk_bounds=2, pairs=3, items=4, slot_offset=5, slot_rows=6,
-              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11, fused_units=12)
-_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, fused_units=16)
+              fwd_units=7, bwd_units=8, bwd_qranges=9, merge_units=10, bwd_work=11, fused_units=12, row_limit=13,
+              first_query=14, span_pairs=15)
+_TABLE_WIDTH = dict(pairs=6, items=8, fwd_units=16, bwd_units=8, bwd_qranges=4, merge_units=4, fused_units=16,
+                    span_pairs=5)
 INFO = dict(T=0, R=1, n_pairs=2, n_items=3, n_fwd_units=4, n_bwd_units=5, n_merge_units=6, B=7, n_merge_multi=8,
             n_fused_units=9)
 
-EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
+EXPORTS = ["fcp_plan_strategy", "fcp_plan_blocks", "fcp_plan_blocks_spans", "fcp_span_mask_efficiency", "fcp_plan_get", "fcp_plan_info", "fcp_plan_workspace_bytes",
            "fcp_plan_bwd_scratch_bytes", "fcp_plan_upload", "fcp_plan_destroy", "fcp_attn_fwd", "fcp_attn_fwd_merged",
            "fcp_attn_fwd_fused", "fcp_lse_merge", "fcp_attn_bwd", "fcp_attn_bwd_heads",
            "fcp_host_workspace_bytes", "fcp_attn_fwd_bwd_host", "fcp_last_device_status", "fcp_plan_set_profiling",
@@ -64,6 +66,8 @@ def lib() -> C.CDLL:
     L.fcp_plan_strategy.argtypes = [i32p, C.c_int32, C.c_int32, C.c_double, C.c_double, C.c_double,
                                     C.POINTER(FcpCostCoeffs), i32p, i32p, i32p, f64p]
     L.fcp_plan_blocks.argtypes = [i32p, i32p, C.c_int32, C.POINTER(FcpParams), C.POINTER(vp)]
+    L.fcp_plan_blocks_spans.argtypes = [i32p, i32p, C.c_int32, i32p, i32p, C.POINTER(FcpParams), C.POINTER(vp)]
+    L.fcp_span_mask_efficiency.argtypes = [C.c_int32, i32p, C.c_int32, f64p]
     L.fcp_plan_get.argtypes = [vp, C.c_int32, C.POINTER(i32p), i64p]
     L.fcp_plan_info.argtypes = [vp, C.c_int32, i64p]
     L.fcp_plan_workspace_bytes.argtypes = [vp, C.c_int32, i64p, i64p, i64p]
@@ -140,14 +144,25 @@ def fcp_plan_strategy(seqlens, N, E, M_token, M_ms, coeffs: dict, eta=None):
 class Plan:
     """Owns an fcp_plan handle."""
 
-    def __init__(self, seqlens, cp_degrees, hq, hkv, head_dim, scale=0.0):
+    def __init__(self, seqlens, cp_degrees, hq, hkv, head_dim, scale=0.0, spans=None):
+        """spans: None, or one list of (begin, end) pairs per sequence (positions relative to its start)."""
         sl, slp = _i32(seqlens)
         dg, dgp = _i32(cp_degrees)
         if len(sl) != len(dg):
             raise ValueError("seqlens and cp_degrees differ in length")
         self.params = FcpParams(int(hq), int(hkv), int(head_dim), float(scale))
         self.handle = C.c_void_p()
-        _check(lib().fcp_plan_blocks(slp, dgp, len(sl), C.byref(self.params), C.byref(self.handle)))
+        if spans is None:
+            _check(lib().fcp_plan_blocks(slp, dgp, len(sl), C.byref(self.params), C.byref(self.handle)))
+        else:
+            if len(spans) != len(sl):
+                raise ValueError("spans needs one list per sequence")
+            off = np.zeros(len(sl) + 1, dtype=np.int32)
+            off[1:] = np.cumsum([len(x) for x in spans])
+            flat = np.asarray([v for x in spans for ab in x for v in ab], dtype=np.int32)
+            so, sop = _i32(off)
+            fl, flp = _i32(flat if flat.size else np.zeros(2, dtype=np.int32))
+            _check(lib().fcp_plan_blocks_spans(slp, dgp, len(sl), sop, flp, C.byref(self.params), C.byref(self.handle)))
         self.hq, self.hkv, self.head_dim = int(hq), int(hkv), int(head_dim)
 
     def __del__(self):
@@ -205,6 +220,19 @@ class Plan:
 
 def fcp_plan_blocks(seqlens, cp_degrees, hq, hkv, head_dim, scale=0.0) -> Plan:
     return Plan(seqlens, cp_degrees, hq, hkv, head_dim, scale)
+
+
+def fcp_plan_blocks_spans(seqlens, cp_degrees, spans, hq, hkv, head_dim, scale=0.0) -> Plan:
+    return Plan(seqlens, cp_degrees, hq, hkv, head_dim, scale, spans=spans)
+
+
+def fcp_span_mask_efficiency(length, spans) -> float:
+    """eta_k of one sequence (Eq. 4): visible pairs over the causal count, minus 1."""
+    flat = np.asarray([v for ab in spans for v in ab], dtype=np.int32)
+    fl, flp = _i32(flat if flat.size else np.zeros(2, dtype=np.int32))
+    eta = C.c_double(0.0)
+    _check(lib().fcp_span_mask_efficiency(int(length), flp, len(spans), C.byref(eta)))
+    return eta.value
 
 
 def fcp_attn_fwd(plan: Plan, q, k, v, o_partial, lse_partial, head_begin=0, head_count=None, stream=0):

@@ -26,7 +26,7 @@ class DeviceState:
         """q, k, v, do: bf16 bit patterns on the host (numpy uint16) or bf16 tensors already on the device.
         `partials=False` skips the partial buffers (enough for the fused forward)."""
         self.w = w
-        self.plan = fcp.fcp_plan_blocks(w.seqlens, w.cp_degrees, w.hq, w.hkv, w.head_dim).upload()
+        self.plan = fcp.Plan(w.seqlens, w.cp_degrees, w.hq, w.hkv, w.head_dim, spans=w.spans).upload()
         T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
         self.hpp = heads_per_pass or hq
         dev = lambda a: a if isinstance(a, torch.Tensor) else to_dev_bf16(a)

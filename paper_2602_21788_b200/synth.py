@@ -70,6 +70,7 @@ class Workload:
     head_dim: int
     note: str = ""
     extra: dict = field(default_factory=dict)
+    spans: list | None = None      # per sequence a list of (begin, end) bidirectional spans, or None (causal)
 
     @property
     def total_tokens(self) -> int:
@@ -88,6 +89,14 @@ class Workload:
     def flops_fwd(self) -> float:
         """Causal forward FLOPs by the headline accounting: 2 * sum L^2 * hq * D."""
         return 2.0 * self.sum_sq * self.hq * self.head_dim
+
+    @property
+    def visible_pairs(self) -> int:
+        """(query, key) pairs the mask keeps: L(L+1)/2 per sequence plus m(m-1)/2 per span of m tokens."""
+        n = int((self.seqlens.astype(np.int64) * (self.seqlens.astype(np.int64) + 1) // 2).sum())
+        for sp in self.spans or []:
+            n += sum((e - a) * (e - a - 1) // 2 for a, e in sp)
+        return n
 
     def flops_fwd_bwd(self) -> float:
         return 3.5 * self.flops_fwd()
@@ -182,12 +191,32 @@ def _extreme_512k(rng, d_long=7):
     return lens, deg, dict(hq=64, hkv=8, head_dim=128)
 
 
+def _bimodal_128k_spans(rng):
+    """The bimodal batch with image spans: every long (image/video-token-heavy) sequence alternates text
+    runs of U{64..512} tokens with bidirectional spans of U{256..2048} tokens; short sequences stay causal."""
+    lens, deg, shape = _bimodal_128k(rng)
+    spans = []
+    for L in lens:
+        sp, pos = [], 0
+        if L >= 16384:
+            while True:
+                pos += int(rng.integers(64, 513))
+                m = int(rng.integers(256, 2049))
+                if pos + m > L:
+                    break
+                sp.append((pos, pos + m))
+                pos += m
+        spans.append(sp)
+    return lens, deg, dict(shape, spans=spans)
+
+
 WORKLOADS = {
     "tiny": _tiny,
     "llama8b_64k": _llama8b_64k,
     "longtail_256k": _longtail_256k,
     "bimodal_128k": _bimodal_128k,
     "extreme_512k": _extreme_512k,
+    "bimodal_128k_spans": _bimodal_128k_spans,
 }
 
 
@@ -205,5 +234,9 @@ def reduced(w: Workload, len_div: int = 16, max_heads: int = 8) -> Workload:
     hq = max(g, (hq // g) * g) if g <= max_heads else g
     hkv = max(1, hq // g)
     lens = np.maximum(1, w.seqlens // len_div).astype(np.int32)
+    spans = None
+    if w.spans is not None:      # span bounds scale with the lengths; spans that collapse are dropped
+        spans = [[(a // len_div, min(e // len_div, int(L))) for a, e in sp if min(e // len_div, int(L)) > a // len_div]
+                 for sp, L in zip(w.spans, lens)]
     return Workload(name=w.name + "_reduced", seed=w.seed, seqlens=lens, cp_degrees=w.cp_degrees.copy(),
-                    hq=hq, hkv=hkv, head_dim=w.head_dim, note=f"lengths/{len_div}")
+                    hq=hq, hkv=hkv, head_dim=w.head_dim, note=f"lengths/{len_div}", spans=spans)

@@ -58,8 +58,9 @@ def test_block_plan_bit_exact_on_workloads(name, seed):
     assert plan.info("T") == w.total_tokens
 
 
-def _cover_fwd(units, T):
-    """Token-pair coverage implied by a table of forward work units (per-item or fused)."""
+def _cover_fwd(units, T, row_limit=None):
+    """Token-pair coverage implied by a table of forward work units (per-item or fused); `row_limit`:
+    the plan's row limits when it has bidirectional spans (a DIAG range then ends at the row's limit)."""
     fwd = np.zeros((T, T), dtype=np.int32)
     for u in units:
         q0, rows, prow, nr = u[0], u[1], u[2], u[3]
@@ -74,11 +75,37 @@ def _cover_fwd(units, T):
                     qp = q0 + 128 * s + row
                     limit = ke - ks
                     if kd:
-                        limit = min(limit, qp - ks + 1)
+                        limit = min(limit, (qp + 1 if row_limit is None else row_limit[qp]) - ks)
                     limit = min(limit, 128)
-                    assert limit >= 1
-                    fwd[qp, ks:ks + limit] += 1
+                    assert limit >= 1 or row_limit is not None
+                    if limit > 0:
+                        fwd[qp, ks:ks + limit] += 1
     return fwd
+
+
+def _cover_bwd(plan, T, first_query=None):
+    """Token-pair coverage implied by the backward units: a DIAG range runs from Q tile T_FIRST on, and the
+    tiles before T_MASK_END drop the queries before each key's first query (the key itself, or its span's begin)."""
+    bwd = np.zeros((T, T), dtype=np.int32)
+    qr = plan.table("bwd_qranges")
+    for u in plan.table("bwd_units"):
+        k0, krows, first, nq, t_first, cost, t_mask_end = u[0], u[1], u[2], u[3], u[4], u[5], u[7]
+        n = 0
+        for r in range(nq):
+            qb, qe, diag = qr[first + r][:3]
+            t = t_first if diag else 0
+            while qb + 128 * t < qe:
+                n += 1
+                q_row = qb + 128 * t
+                qv = min(128, qe - q_row)
+                for row in range(krows):
+                    fq = k0 + row if first_query is None else first_query[k0 + row]
+                    lo = max(0, fq - q_row) if (diag and t < t_mask_end) else 0
+                    if lo < qv:
+                        bwd[q_row + lo:q_row + qv, k0 + row] += 1
+                t += 1
+        assert n == cost
+    return bwd
 
 
 def _cover(plan, lens):
@@ -86,23 +113,7 @@ def _cover(plan, lens):
     cu = np.concatenate([[0], np.cumsum(lens)])
     T = int(cu[-1])
     fwd = _cover_fwd(plan.table("fwd_units"), T)
-    bwd = np.zeros((T, T), dtype=np.int32)
-    qr = plan.table("bwd_qranges")
-    for u in plan.table("bwd_units"):
-        k0, krows, first, nq, ktile, cost = u[0], u[1], u[2], u[3], u[4], u[5]
-        n = 0
-        for r in range(nq):
-            qb, qe, diag = qr[first + r][:3]
-            t = ktile if diag else 0
-            while qb + 128 * t < qe:
-                n += 1
-                q_row = qb + 128 * t
-                qv = min(128, qe - q_row)
-                for row in range(krows):
-                    lo = max(0, k0 + row - q_row) if (diag and t == ktile) else 0
-                    bwd[q_row + lo:q_row + qv, k0 + row] += 1
-                t += 1
-        assert n == cost
+    bwd = _cover_bwd(plan, T)
     want = np.zeros((T, T), dtype=np.int32)
     for b in range(len(lens)):
         L = lens[b]
@@ -236,3 +247,53 @@ def test_error_paths():
     assert e.value.status == fcp.FCP_ERR_NOT_UPLOADED
     a, b, c = plan.workspace_bytes(8)
     assert a == plan.info("R") * 8 * 128 * 4 and b == plan.info("R") * 8 * 4 and c > 10 * 8 * 128 * 4
+
+
+# ----------------------------------------------------------------------------------------------
+# bidirectional spans
+# ----------------------------------------------------------------------------------------------
+SPAN_CASES = [
+    ([300], [1], [[(100, 140)]]),                                   # inside one tile boundary region
+    ([300], [1], [[(120, 135), (250, 300)]]),                       # across a tile edge; up to the sequence end
+    ([700, 50], [3, 2], [[(0, 130), (230, 236), (400, 699)], []]),  # across chunk edges (bounds 116, 233, 350, ...)
+    ([1030], [6], [[(80, 95), (500, 860)]]),                        # a span over several chunks
+    ([257, 129], [1, 1], [[(0, 257)], [(1, 2)]]),                   # whole sequence; a one-token span (no effect)
+]
+
+
+@pytest.mark.parametrize("lens,degs,spans", SPAN_CASES)
+def test_span_plan_tables_bit_exact_and_units_cover_the_mask(lens, degs, spans):
+    from oracle import span_attention_ref as S
+    plan = fcp.fcp_plan_blocks_spans(lens, degs, spans, 4, 2, 128)
+    ref = P.span_tables(lens, degs, spans)
+    assert plan.table("row_limit").tolist() == ref["row_limit"]
+    assert plan.table("first_query").tolist() == ref["first_query"]
+    assert plan.table("span_pairs").tolist() == [list(x) for x in ref["span_pairs"]]
+    _compare(plan, P.plan_blocks(lens, degs))                       # the causal tables are unchanged
+    T = sum(lens)
+    want = np.zeros((T, T), dtype=np.int32)
+    t0 = 0
+    for b, L in enumerate(lens):
+        lim = S.row_limits(L, spans[b])
+        for i in range(L):
+            want[t0 + i, t0:t0 + lim[i]] = 1
+        t0 += L
+    assert np.array_equal(_cover_fwd(plan.table("fused_units"), T, plan.table("row_limit")), want)
+    assert np.array_equal(_cover_bwd(plan, T, plan.table("first_query")), want)
+    for b, L in enumerate(lens):
+        assert math.isclose(fcp.fcp_span_mask_efficiency(L, spans[b]), S.mask_efficiency(L, spans[b]), rel_tol=1e-12)
+
+
+def test_span_plan_without_spans_is_the_causal_plan_and_bad_spans_are_refused():
+    a = fcp.fcp_plan_blocks([500, 77], [2, 1], 4, 4, 64)
+    b = fcp.fcp_plan_blocks_spans([500, 77], [2, 1], [[], []], 4, 4, 64)
+    for name in ("pairs", "items", "fwd_units", "fused_units", "bwd_units", "bwd_qranges", "bwd_work", "merge_units"):
+        assert np.array_equal(a.table(name), b.table(name)), name
+    assert b.table("row_limit").size == 0 and b.table("span_pairs").size == 0
+    for bad in ([[(5, 5)], []], [[(10, 600)], []], [[(20, 30), (25, 40)], []], [[(30, 40), (10, 20)], []], [[(-1, 4)], []]):
+        with pytest.raises(fcp.FcpError) as e:
+            fcp.fcp_plan_blocks_spans([500, 77], [2, 1], bad, 4, 4, 64)
+        assert e.value.status == fcp.FCP_ERR_INVALID_ARG
+    with pytest.raises(fcp.FcpError) as e:
+        fcp.fcp_span_mask_efficiency(10, [(3, 30)])
+    assert e.value.status == fcp.FCP_ERR_INVALID_ARG
