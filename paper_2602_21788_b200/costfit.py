@@ -18,7 +18,7 @@ import argparse
 import numpy as np
 
 # Last fit on a B200 (32 query / 8 KV heads, head_dim 128), ms units; see `main` for how it is taken.
-B200_COEFFS = dict(alpha1=3.304068e-08, alpha2=1.535782e-06, beta1=1.788982e-02)
+B200_COEFFS = dict(alpha1=2.968323e-08, alpha2=1.505158e-05, beta1=2.173566e-04)
 
 
 def design_row(seqlens, cp_degrees):

@@ -121,38 +121,52 @@ extern "C" int fcp_plan_strategy(const int32_t* seqlens, int32_t B, int32_t N, d
     g.tot += L;
   }
 
-  // Stage 2: Algorithm 1.  Only DP[0][0] is finite initially; strict '<' keeps the smallest d on ties.
+  // Stage 2: the recurrence of Eq. 7, best[k][j] = min over d of max(best[k-1][j-d], T(G_k, d)), kept as two
+  // rolling rows over j plus the arg-min of every (group, j) cell for the walk back.  A cell (k, j) is
+  // reachable when the first k groups can have their minimum degrees (j >= lo[k]) and the remaining ones
+  // still get theirs (j <= N - (need - lo[k])); d ranges over [d_min, j - lo[k-1]].  Ties keep the smallest
+  // d (strict comparison, d ascending).  The answer is read at j = N: the strategy hands out every rank, as
+  // the paper's text does ("backtrack from DP[K'][N]"; its case-study mixes add up to the rank count).
+  // Because T(G, d) is not monotone in d once the ring term appears at d = 2, a plan that leaves ranks
+  // idle could have a smaller makespan; that variant (min over j <= N) is not what the paper runs.
   const double INF = std::numeric_limits<double>::infinity();
-  std::vector<double> dp((size_t)(K + 1) * (N + 1), INF);
-  std::vector<int> path((size_t)(K + 1) * (N + 1), 0);
-  auto at = [&](int k, int j) -> size_t { return (size_t)k * (N + 1) + j; };
-  dp[at(0, 0)] = 0.0;
-  int before = 0;                       // sum of d_min of groups 1..k-1
-  int remain = (int)need_ranks;         // sum of d_min of groups k+1..K'
-  for (int k = 1; k <= K; ++k) {
-    remain -= dmin[k - 1];
-    for (int j = before + dmin[k - 1]; j <= N - remain; ++j) {
-      for (int d = dmin[k - 1]; d <= j - before; ++d) {
-        const double cost = std::max(dp[at(k - 1, j - d)], group_time(sums[k - 1], d, *coeffs));
-        if (cost < dp[at(k, j)]) {
-          dp[at(k, j)] = cost;
-          path[at(k, j)] = d;
+  std::vector<int> lo(K + 1, 0);                 // lo[k] = sum of d_min over the first k groups
+  for (int k = 0; k < K; ++k) lo[k + 1] = lo[k] + dmin[k];
+  std::vector<double> prev(N + 1, INF), cur(N + 1, INF);
+  std::vector<int> choice((size_t)K * (N + 1), 0);
+  std::vector<double> tg(N + 1, 0.0);            // T(G_k, d) for the group at hand
+  prev[0] = 0.0;
+  for (int k = 0; k < K; ++k) {
+    const int j_hi = N - ((int)need_ranks - lo[k + 1]);
+    for (int d = dmin[k]; d <= j_hi - lo[k]; ++d) tg[d] = group_time(sums[k], d, *coeffs);
+    std::fill(cur.begin(), cur.end(), INF);
+    for (int j = lo[k + 1]; j <= j_hi; ++j) {
+      double best = INF;
+      int arg = 0;
+      for (int d = dmin[k]; d <= j - lo[k]; ++d) {
+        const double cand = std::max(prev[j - d], tg[d]);
+        if (cand < best) {
+          best = cand;
+          arg = d;
         }
       }
+      cur[j] = best;
+      choice[(size_t)k * (N + 1) + j] = arg;
     }
-    before += dmin[k - 1];
+    prev.swap(cur);
   }
+  const double best_makespan = prev[N];
   std::vector<int> deg(K, 0);
-  for (int p = K, q = N; p > 0; --p) {
-    deg[p - 1] = path[at(p, q)];
-    q -= deg[p - 1];
+  for (int k = K - 1, j = N; k >= 0; --k) {
+    deg[k] = choice[(size_t)k * (N + 1) + j];
+    j -= deg[k];
   }
   for (int i = 0; i < B; ++i) {
     if (group_of) group_of[i] = gof[i];
     if (cp_degree) cp_degree[i] = deg[gof[i]];
   }
   if (n_groups) *n_groups = K;
-  if (makespan) *makespan = dp[at(K, N)];
+  if (makespan) *makespan = best_makespan;
   return FCP_OK;
 }
 
