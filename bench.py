@@ -32,7 +32,7 @@ sys.path.insert(0, ROOT)
 
 METRIC = "fwd+bwd attention TFLOPS/GPU on packed varlen batches"
 NOMINAL_BF16_TFLOPS = 2250.0      # vendor's public dense BF16 figure, for context only
-OTHER_WORKLOADS = ("longtail_256k", "bimodal_128k")
+OTHER_WORKLOADS = ("longtail_256k", "bimodal_128k", "bimodal_128k_spans")
 KERNEL_KINDS = ["attn_fwd", "lse_merge", "bwd_preprocess", "attn_bwd", "dq_convert"]
 
 # DRAM bytes (read + write) of one backward-kernel launch, from an ncu capture (`profiles/`) of a cut of the
@@ -72,7 +72,8 @@ def config_of(w, seed):
     return {"workload": w.name, "tokens": w.total_tokens, "sequences": int(len(w.seqlens)), "hq": w.hq, "hkv": w.hkv,
             "head_dim": w.head_dim, "seed": seed, "sum_len_sq": w.sum_sq,
             "cp_degrees": sorted(set(int(x) for x in w.cp_degrees)),
-            "flops": "7 * sum(L^2) * hq * head_dim per step"}
+            "spans": sum(len(x) for x in w.spans) if w.spans else 0,
+            "flops": "7 * sum(L^2) * hq * head_dim per step" + (" (+ 14 * hq * head_dim per pair a span adds)" if w.spans else "")}
 
 
 # --------------------------------------------------------------------------------------------

@@ -87,8 +87,10 @@ class Workload:
         return int((self.seqlens.astype(np.int64) ** 2).sum())
 
     def flops_fwd(self) -> float:
-        """Causal forward FLOPs by the headline accounting: 2 * sum L^2 * hq * D."""
-        return 2.0 * self.sum_sq * self.hq * self.head_dim
+        """Forward FLOPs by the headline accounting: 2 * sum L^2 * hq * D for a causal batch (4 * D per
+        (query, key) pair over L^2 / 2 pairs); a span of m tokens adds its m(m-1)/2 pairs above the diagonal."""
+        extra = sum((e - a) * (e - a - 1) // 2 for sp in (self.spans or []) for a, e in sp)
+        return (2.0 * self.sum_sq + 4.0 * extra) * self.hq * self.head_dim
 
     @property
     def visible_pairs(self) -> int:
