@@ -35,10 +35,15 @@ NOMINAL_BF16_TFLOPS = 2250.0      # vendor's public dense BF16 figure, for conte
 OTHER_WORKLOADS = ("longtail_256k", "bimodal_128k", "bimodal_128k_spans")
 KERNEL_KINDS = ["attn_fwd", "lse_merge", "bwd_preprocess", "attn_bwd", "dq_convert"]
 
-# DRAM bytes (read + write) of one backward-kernel launch, from an ncu capture (`profiles/`) of a cut of the
-# workload to `heads` query heads, scaled to all heads by the (unit, KV head) work items processed; with the
-# digest of the sources that decide the kernel and its work order: reported only while they still match.
+# DRAM bytes (read + write) of one backward-kernel launch of the timed workload from an ncu capture, with the digest
+# of the sources that decide the kernel and its work order: reported only while they still match.  The bench
+# workload has no entry: its launch runs for seconds and the DRAM counters take several passes, which the capture
+# rules of the GPU pool keep to small cases; the traffic of a launch does not scale from a small case in proportion
+# (it depends on what stays in L2), so `roofline.traffic` is null and the small-case capture is reported beside it.
 NCU_BWD_TRAFFIC = {}
+NCU_BWD_TRAFFIC_SMALL_CASE = {
+    "workload": "longtail_256k cut to 5 query heads on 1 KV head", "traffic": 4035786000 + 2922308000,
+    "algorithmic_bytes": 2282000000, "ms": 52.8, "summary": "profiles/bwd_kernel_longtail_256k_5heads.md"}
 
 
 def bwd_kernel_digest():
@@ -195,6 +200,12 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------
 # our arm
 # --------------------------------------------------------------------------------------------
+def per_ghz(tflops, clocks):
+    """Clock-normalised throughput: TFLOPS per GHz of the median SM clock sampled during the timed region."""
+    mhz = (clocks or {}).get("sm_mhz")
+    return tflops / (mhz / 1000.0) if mhz else None
+
+
 def time_planner(w, reps=20):
     """Host time of the two planner calls alone (no CUDA call inside the timers), microseconds."""
     from paper_2602_21788_b200 import costfit, fcp
@@ -418,6 +429,7 @@ def run_ours(args, w):
               else "sustained figure (seconds under the power cap, clock well below maximum)"))
     roofline = {"bound": "tensor", "kernel": "fcp_bwd_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                 "frac": achieved / peak if achieved else None, "traffic": ncu_traffic(w, args),
+                "traffic_small_case": NCU_BWD_TRAFFIC_SMALL_CASE,
                 "flops_per_launch": bwd_flops, "ms_per_launch": bwd_ms,
                 "peak_source": f"{peaks['source']} {'burst' if use_burst else 'sustained'} bf16 cuBLAS; {why}",
                 "fwd_kernel": {"achieved": w.flops_fwd() / (fwd_ms * 1e-3) / 1e12 if fwd_ms > 0 else None, "ms": fwd_ms,
@@ -442,7 +454,8 @@ def run_ours(args, w):
                 "attn_fwd_tflops": ow.flops_fwd() / (k2["attn_fwd"]["mean_ms"] * 1e-3) / 1e12,
                 "attn_bwd_tflops": 2.5 * ow.flops_fwd() / (k2["attn_bwd"]["mean_ms"] * 1e-3) / 1e12,
                 "frac_of_burst": r["value"] / peaks["bf16_burst"], "frac_of_sustained": r["value"] / peaks["bf16_sustained"],
-                "frac_of_vendor_dense_bf16": r["value"] / NOMINAL_BF16_TFLOPS, "clocks": r["clocks"]}
+                "frac_of_vendor_dense_bf16": r["value"] / NOMINAL_BF16_TFLOPS, "clocks": r["clocks"],
+                "tflops_per_sm_ghz": per_ghz(r["value"], r["clocks"])}
             del r
             torch.cuda.empty_cache()
     if sampler:
@@ -469,6 +482,7 @@ def run_ours(args, w):
                          "vendor_dense_bf16": value / world / NOMINAL_BF16_TFLOPS},
         "kernels": kern, "roofline": roofline, "partial_path": main.get("partial_path"), "other_workloads": others,
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": args.steps * (passes + 3), "clocks": clocks,
+        "tflops_per_sm_ghz": per_ghz(value / world, clocks),
     }
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -529,7 +543,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-other-workloads", action="store_true")
-    ap.add_argument("--other-steps", type=int, default=6, help="timed steps of each workload under other_workloads")
+    ap.add_argument("--other-steps", type=int, default=10, help="timed steps of each workload under other_workloads")
     ap.add_argument("--no-partial-path", action="store_true")
     ap.add_argument("--heads-per-pass", type=int, default=0, help="query heads per forward pass (0 = all)")
     ap.add_argument("--max-heads", type=int, default=0,
