@@ -686,9 +686,9 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
     b0 = b1;
   }
   tok0.push_back(T);
-  // streams and events: [0] start, [1] last copy out, then per group (inputs up, kernels done)
+  // streams and events: [0] start, [1] last copy out, then per group (q, k, v up; dO up; forward done; backward done)
   cudaStream_t in = nullptr, out = nullptr;
-  std::vector<void*> ev(2 + 2 * groups.size(), nullptr);
+  std::vector<void*> ev(2 + 4 * groups.size(), nullptr);
   cudaError_t e = cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking);
   for (size_t i = 0; i < ev.size() && e == cudaSuccess; ++i) {
@@ -753,35 +753,43 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   // complete when this call returns.
   cudaStream_t s_in = (cudaStream_t)plan->host_in, s_out = (cudaStream_t)plan->host_out;
   auto EV = [&](int i) { return (cudaEvent_t)plan->host_events[i]; };
-  auto ev_up = [&](int g) { return EV(2 + 2 * g); };
-  auto ev_done = [&](int g) { return EV(3 + 2 * g); };
+  auto ev_qkv = [&](int g) { return EV(2 + 4 * g); };
+  auto ev_do = [&](int g) { return EV(3 + 4 * g); };
+  auto ev_fwd = [&](int g) { return EV(4 + 4 * g); };
+  auto ev_bwd = [&](int g) { return EV(5 + 4 * g); };
   HostDrain drain{s_in, s_out, st};
   FCP_CUDA_CHECK(cudaEventRecord(EV(0), st));
   FCP_CUDA_CHECK(cudaStreamWaitEvent(s_in, EV(0), 0));
   FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, EV(0), 0));
+  // The forward pass of a run needs q, k, v only: dO follows them and arrives while the forward kernel runs;
+  // o and lse leave while the backward kernels run (they only read them).
   for (int g = 0; g < G; ++g) {
     const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
     FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q + t0 * rq, (const char*)q_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
     FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k + t0 * rkv, (const char*)k_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
     FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v + t0 * rkv, (const char*)v_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaEventRecord(ev_qkv(g), s_in));
     FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o + t0 * rq, (const char*)d_o_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
-    FCP_CUDA_CHECK(cudaEventRecord(ev_up(g), s_in));
+    FCP_CUDA_CHECK(cudaEventRecord(ev_do(g), s_in));
   }
   for (int g = 0; g < G; ++g) {
     const fcp_plan* sub = plan->groups[g];
     const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_up(g), 0));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_qkv(g), 0));
     if ((rc = fcp_attn_fwd_fused(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, 0, P.hq, w + L.o + t0 * rq,
                                  nullptr, (float*)(w + L.lse + t0 * rl), st)) != FCP_OK)
       return rc;
+    FCP_CUDA_CHECK(cudaEventRecord(ev_fwd(g), st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_fwd(g), 0));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_do(g), 0));
     if ((rc = fcp_attn_bwd(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, w + L.o + t0 * rq,
                            w + L.d_o + t0 * rq, (float*)(w + L.lse + t0 * rl), w + L.dq + t0 * rq, w + L.dk + t0 * rkv,
                            w + L.dv + t0 * rkv, w + L.scratch, bwd_scratch_need(sub, P.hkv), st)) != FCP_OK)
       return rc;
-    FCP_CUDA_CHECK(cudaEventRecord(ev_done(g), st));
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_done(g), 0));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaEventRecord(ev_bwd(g), st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_bwd(g), 0));
     FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dq_host + t0 * rq, w + L.dq + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
     FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dk_host + t0 * rkv, w + L.dk + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));
     FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dv_host + t0 * rkv, w + L.dv + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));

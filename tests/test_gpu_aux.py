@@ -64,3 +64,33 @@ def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable():
     dq_ref, dk_ref, dv_ref = A.attention_bwd_packed(f(q), f(k), f(v), f(do), w.cu_seqlens)
     for name, ref in (("dq", dq_ref), ("dk", dk_ref), ("dv", dv_ref)):
         assert np.linalg.norm(res[name] - ref) <= 2e-2 * np.linalg.norm(ref)
+
+
+def test_no_call_writes_outside_the_buffers_it_was_given():
+    """Guard bands around every output and workspace buffer (64 KB of a byte pattern on both sides) stay
+    untouched by the partial path, the merged and the fused forward and the backward pass, on a ragged batch
+    (tiles cut by sequence ends, empty chunks, head passes)."""
+    from paper_2602_21788_b200.runner import DeviceState
+    GUARD = 1 << 16
+    w = synth.Workload(name="guards", seed=6, seqlens=np.asarray([1, 700, 129, 3, 1031], np.int32),
+                       cp_degrees=np.asarray([1, 3, 1, 4, 5], np.int32), hq=4, hkv=2, head_dim=128)
+    q, k, v, do = w.tensors()
+    ds = DeviceState(w, q, k, v, do, heads_per_pass=3, want_o_f32=True, kv_heads_per_bwd_pass=1)
+    arenas = {}
+    for name in ("o_part", "lse_part", "o", "lse", "o_f32", "dq", "dk", "dv", "scratch"):
+        t = getattr(ds, name)
+        nbytes = t.numel() * t.element_size()
+        arena = torch.full((nbytes + 2 * GUARD,), 0xA5, dtype=torch.uint8, device="cuda")
+        inner = arena[GUARD:GUARD + nbytes].view(t.dtype).view(t.shape)
+        assert inner.data_ptr() % 256 == 0
+        setattr(ds, name, inner)
+        arenas[name] = (arena, nbytes)
+    ds.forward()
+    ds.forward(merged=True)
+    ds.forward_fused()
+    ds.backward()
+    torch.cuda.synchronize()
+    ds.check_status()
+    for name, (arena, nbytes) in arenas.items():
+        assert bool((arena[:GUARD] == 0xA5).all()) and bool((arena[GUARD + nbytes:] == 0xA5).all()), name
+    assert torch.isfinite(ds.o.float()).all() and torch.isfinite(ds.dq.float()).all()
