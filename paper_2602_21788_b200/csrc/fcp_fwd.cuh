@@ -49,6 +49,9 @@ struct FwdArgs {
   int32_t head_begin, head_count, hq, hkv;
   int32_t head_group;     // heads that are adjacent in the work order: hq/hkv when the head range is made of whole
                           // KV-head groups, else 1; head_count % head_group == 0
+  int32_t round_heads;    // heads per round group (a multiple of head_group): rounds never mix two round groups
+  int32_t* round_counter; // nullptr, or a zeroed counter: the CTAs meet (for at most round_sync_ns) at every round start
+  uint32_t round_sync_ns;
   float scale_log2;       // softmax scale * log2(e)
   float* o_partial;       // [R][head_count][D]
   float* lse_partial;     // [R][head_count]
@@ -116,23 +119,31 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   const int64_t n_work = (int64_t)a.n_units * a.head_count;
   const int g = a.hq / a.hkv;
-  // Work item w = (head within an inner group of `gi` heads, unit, group), innermost first: with gi =
-  // the query heads of one KV head, the CTAs that run at the same time work on adjacent units of the
-  // same KV head and stream the same K/V tiles (one copy in L2 serves them all).  CTA c takes the
-  // items c, 2G-1-c, 2G+c, ... (G = grid size): units are sorted by cost, so alternating the
-  // direction of every other round evens out the systematic bias of a fixed stride.  Every role
-  // walks the same sequence.
+  // Work order.  The heads of the pass are cut into round groups of `round_heads` heads (whole KV-head groups
+  // when the head range allows it: gi = query heads per KV head, else gi = 1).  Inside a round group the items
+  // are ordered (head within its KV group, unit, KV head), innermost first, and dealt out in rounds of G = grid
+  // size items: CTA c takes position c of the even rounds and G-1-c of the odd ones (units are sorted by cost,
+  // so alternating the direction evens out the bias of a fixed stride).  The CTAs that run at the same time thus
+  // work on adjacent units of the same KV head and stream the same K/V tiles: one copy in L2 serves them all.
+  // A round never mixes two round groups, so all its items cost about the same and the CTAs stay in step.
+  // Every role walks the same sequence.
   const int gi = a.head_group;
+  const int64_t G = gridDim.x;
+  const int64_t rpg = ((int64_t)a.n_units * a.round_heads + G - 1) / G;      // rounds per (full) round group
+  const int n_round_groups = (a.head_count + a.round_heads - 1) / a.round_heads;
+  const int last_heads = a.head_count - (n_round_groups - 1) * a.round_heads;   // the last group may be smaller
   auto work_item = [&](int64_t round, const int32_t*& U, int& h) -> bool {
-    const int64_t G = gridDim.x;
-    const int64_t w = round * G + ((round & 1) ? G - 1 - (int64_t)blockIdx.x : (int64_t)blockIdx.x);
-    if (w >= n_work) return false;          // only in the last round
-    const int64_t grp = w / gi;
-    U = a.units + (size_t)(grp % a.n_units) * FCP_FWD_UNIT_W;
-    h = a.head_begin + (int)(grp / a.n_units) * gi + (int)(w % gi);
+    const int gidx = (int)min(round / rpg, (int64_t)(n_round_groups - 1));
+    const int64_t rr = round - (int64_t)gidx * rpg;
+    const int64_t idx = rr * G + ((rr & 1) ? G - 1 - (int64_t)blockIdx.x : (int64_t)blockIdx.x);
+    const int hcnt = min(a.round_heads, a.head_count - gidx * a.round_heads);
+    if (idx >= (int64_t)a.n_units * hcnt) return false;       // padding at the end of a round group
+    const int64_t t = idx / gi;
+    U = a.units + (size_t)(t % a.n_units) * FCP_FWD_UNIT_W;
+    h = a.head_begin + gidx * a.round_heads + (int)(t / a.n_units) * gi + (int)(idx % gi);
     return true;
   };
-  const int64_t n_rounds = (n_work + gridDim.x - 1) / gridDim.x;
+  const int64_t n_rounds = rpg * (n_round_groups - 1) + ((int64_t)a.n_units * last_heads + G - 1) / G;
 
   if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_CTRL ";");
   if (warp == 0) {
@@ -141,7 +152,24 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       uint32_t kv_it = 0, qcnt[2] = {0, 0};
       bool ok = true;
 #pragma unroll 1
+      uint32_t sync_misses = 0;
       for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+        // Meeting point of the grid at the start of a round.  When one KV head's keys and values exceed the L2
+        // the CTAs only share K/V tiles while they sweep them in step; small differences in speed add up over
+        // hundreds of rounds, so they wait for each other here.  The wait is advisory: nothing depends on it,
+        // it ends after round_sync_ns whoever is missing, and a CTA that ran out of patience four times stops
+        // waiting for the rest of the launch.
+        if (a.round_counter != nullptr && sync_misses < 4) {
+          atomicAdd(a.round_counter, 1);
+          const int target = (int)((rnd + 1) * G);
+          const uint32_t t0 = globaltimer_lo();
+          bool met = true;
+          while (*(volatile int32_t*)a.round_counter < target) {
+            if (globaltimer_lo() - t0 > a.round_sync_ns) { met = false; break; }
+            __nanosleep(200);
+          }
+          if (!met) ++sync_misses;
+        }
         const int32_t* U;
         int h;
         if (!work_item(rnd, U, h)) continue;

@@ -209,6 +209,7 @@ extern "C" int fcp_plan_blocks_spans(const int32_t* seqlens, const int32_t* cp_d
     return FCP_ERR_UNSUPPORTED;
   }
   int64_t T = 0;
+  int32_t max_len = 0;
   for (int b = 0; b < B; ++b) {
     if (seqlens[b] <= 0 || cp_degrees[b] <= 0) {
       fcp_set_error("fcp_plan_blocks: sequence %d has length %d, degree %d", b, seqlens[b], cp_degrees[b]);
@@ -219,6 +220,7 @@ extern "C" int fcp_plan_blocks_spans(const int32_t* seqlens, const int32_t* cp_d
       return FCP_ERR_UNSUPPORTED;
     }
     T += seqlens[b];
+    max_len = std::max(max_len, seqlens[b]);
   }
   if (T >= (int64_t(1) << 31) - 2 * FCP_FWD_UNIT_ROWS) {
     fcp_set_error("fcp_plan_blocks: %lld tokens exceed the 2^31 limit", (long long)T);
@@ -230,6 +232,7 @@ extern "C" int fcp_plan_blocks_spans(const int32_t* seqlens, const int32_t* cp_d
   if (!(p->params.scale > 0.f)) p->params.scale = 1.0f / std::sqrt((float)params->head_dim);
   p->B = B;
   p->T = T;
+  p->max_seqlen = max_len;
   p->cu_seqlens.assign(B + 1, 0);
   for (int b = 0; b < B; ++b) p->cu_seqlens[b + 1] = p->cu_seqlens[b] + seqlens[b];
 

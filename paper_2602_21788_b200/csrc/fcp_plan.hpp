@@ -28,6 +28,7 @@ struct fcp_plan {
   fcp_params params{};
   int32_t B = 0;
   int64_t T = 0;   // total tokens
+  int32_t max_seqlen = 0;
   int64_t R = 0;   // rows of the partial buffers
   int32_t n_merge_multi = 0;   // merge units of chunks with two or more slots (they come first in merge_units)
   std::vector<int32_t> cu_seqlens, chunk_offset, chunk_bounds, pairs, items, slot_offset, slot_rows;
