@@ -36,10 +36,10 @@ OTHER_WORKLOADS = ("longtail_256k", "bimodal_128k", "bimodal_128k_spans")
 KERNEL_KINDS = ["attn_fwd", "lse_merge", "bwd_preprocess", "attn_bwd", "dq_convert"]
 
 # DRAM bytes (read + write) of one backward-kernel launch of the timed workload from an ncu capture, with the digest
-# of the sources that decide the kernel and its work order: reported only while they still match.  The bench
-# workload has no entry: its launch runs for seconds and the DRAM counters take several passes, which the capture
-# rules of the GPU pool keep to small cases; the traffic of a launch does not scale from a small case in proportion
-# (it depends on what stays in L2), so `roofline.traffic` is null and the small-case capture is reported beside it.
+# of the sources that decide the kernel and its work order: reported only while they still match.  The default
+# workload has no entry: its launch runs for seconds and the DRAM counters take several replay passes, so it is
+# captured on a small case only; the traffic of a launch does not scale from a small case in proportion (it depends
+# on what stays in L2), so `roofline.traffic` is null and the small-case capture is reported beside it.
 NCU_BWD_TRAFFIC = {}
 NCU_BWD_TRAFFIC_SMALL_CASE = {
     "workload": "longtail_256k cut to 5 query heads on 1 KV head", "traffic": 4035786000 + 2922308000,
@@ -395,7 +395,23 @@ def run_ours(args, w):
 
     # ---- end to end from pinned host buffers through the host entry point
     e2e = None
-    if not args.no_e2e:
+    # every rank of this node pins its own host copies of all inputs and outputs: leave the leg out (on all ranks
+    # alike, it contains a reduction) rather than exhaust the host memory when N batches of this size do not fit
+    pinned_need = world * (8 * w.total_tokens * (w.hq + w.hkv) * w.head_dim + 4 * w.total_tokens * w.hq)
+    host_ok = True
+    try:
+        import psutil
+        host_ok = pinned_need <= 0.6 * psutil.virtual_memory().available
+    except Exception:
+        pass
+    if world > 1:
+        flag = torch.tensor([1 if host_ok else 0], device="cuda")
+        dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+        host_ok = bool(flag.item())
+    if not args.no_e2e and not host_ok:
+        e2e = {"value": None, "unit": "TFLOPS", "skipped": "pinned host buffers of %d ranks (%.0f GB) exceed the host memory"
+               % (world, pinned_need / 1e9)}
+    if not args.no_e2e and host_ok:
         n_e2e = max(1, min(args.steps, args.e2e_steps))
         e_ms, h2d, d2h = run_e2e(w, ds, n_e2e, barrier)
         e_ms, _ = ranks.aggregate(e_ms, 0.0, "cuda")
