@@ -22,6 +22,7 @@ namespace fcp {
 
 constexpr int FWD_THREADS = 512;          // 4 control warps + 2 x 4 softmax warps + 4 epilogue warps
 constexpr int FWD_KV_SLOTS = 4;
+constexpr int FWD_WORK_SLOTS = 4;         // ring of work items handed from the producer to the other roles
 // register budgets per thread of the three roles: 128 * 64 + 256 * 184 + 128 * 80 = 512 * 128
 #define FCP_FWD_REGS_CTRL "64"
 #define FCP_FWD_REGS_SOFTMAX "184"
@@ -36,9 +37,10 @@ struct FwdSmem {
   static constexpr int BAR_OFF = KV_OFF + FWD_KV_SLOTS * KV_TILE_BYTES;
   // barriers: q_full[2] q_empty[2] kv_full[S] kv_empty[S] s_full[2] p_full[2] o_final[2] o_empty[2] turn[2]
   //           stat_full[2] stat_empty[2]
-  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 14;
-  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;   // tmem base (4 B), abort flag (4 B)
-  static constexpr int STAT_OFF = MISC_OFF + 16;          // [2 tiles][row sum, reference maximum][128 rows] fp32
+  //           w_full[W] w_empty[W]
+  static constexpr int N_BARS = 4 + 2 * FWD_KV_SLOTS + 14 + 2 * FWD_WORK_SLOTS;
+  static constexpr int MISC_OFF = BAR_OFF + N_BARS * 8;   // tmem base (4 B), abort flag (4 B), work ring [W][unit, head]
+  static constexpr int STAT_OFF = MISC_OFF + 16 + 8 * FWD_WORK_SLOTS;   // [2 tiles][row sum, reference maximum][128 rows] fp32
   static constexpr int TOTAL = STAT_OFF + 2 * 2 * 128 * 4;
   static constexpr int DYN_BYTES = TOTAL + 1024;          // slack to align the base to 1024 B
 };
@@ -49,9 +51,7 @@ struct FwdArgs {
   int32_t head_begin, head_count, hq, hkv;
   int32_t head_group;     // heads that are adjacent in the work order: hq/hkv when the head range is made of whole
                           // KV-head groups, else 1; head_count % head_group == 0
-  int32_t round_heads;    // heads per round group (a multiple of head_group): rounds never mix two round groups
-  int32_t* round_counter; // nullptr, or a zeroed counter: the CTAs meet (for at most round_sync_ns) at every round start
-  uint32_t round_sync_ns;
+  int32_t* work_counter;  // zero before the launch: the grid's next work item
   float scale_log2;       // softmax scale * log2(e)
   float* o_partial;       // [R][head_count][D]
   float* lse_partial;     // [R][head_count]
@@ -79,9 +79,11 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
   const int B_QFULL = 0, B_QEMPTY = 2, B_KVFULL = 4, B_KVEMPTY = 4 + FWD_KV_SLOTS,
             B_SFULL = 4 + 2 * FWD_KV_SLOTS, B_PFULL = B_SFULL + 2, B_OFINAL = B_SFULL + 4, B_OEMPTY = B_SFULL + 6,
-            B_TURN = B_SFULL + 8, B_STATFULL = B_SFULL + 10, B_STATEMPTY = B_SFULL + 12;
+            B_TURN = B_SFULL + 8, B_STATFULL = B_SFULL + 10, B_STATEMPTY = B_SFULL + 12, B_WFULL = B_SFULL + 14,
+            B_WEMPTY = B_WFULL + FWD_WORK_SLOTS;
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(smem + SM::MISC_OFF);
   volatile int* abort_flag = (volatile int*)(smem + SM::MISC_OFF + 4);
+  volatile int* work_ring = (volatile int*)(smem + SM::MISC_OFF + 16);   // [FWD_WORK_SLOTS][unit, head]
   const WaitCtx wctx{abort_flag, a.status, (uint32_t)FCP_WAIT_NS};
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -98,6 +100,10 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       mbar_init(BAR(B_TURN + i), 4);
       mbar_init(BAR(B_STATFULL + i), 4);
       mbar_init(BAR(B_STATEMPTY + i), 4);
+    }
+    for (int i = 0; i < FWD_WORK_SLOTS; ++i) {
+      mbar_init(BAR(B_WFULL + i), 1);
+      mbar_init(BAR(B_WEMPTY + i), 2 + 8 + 4);   // two issuing threads, one lane of each softmax and epilogue warp
     }
     for (int i = 0; i < FWD_KV_SLOTS; ++i) {
       mbar_init(BAR(B_KVFULL + i), 1);
@@ -119,60 +125,57 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   const int64_t n_work = (int64_t)a.n_units * a.head_count;
   const int g = a.hq / a.hkv;
-  // Work order.  The heads of the pass are cut into round groups of `round_heads` heads (whole KV-head groups
-  // when the head range allows it: gi = query heads per KV head, else gi = 1).  Inside a round group the items
-  // are ordered (head within its KV group, unit, KV head), innermost first, and dealt out in rounds of G = grid
-  // size items: CTA c takes position c of the even rounds and G-1-c of the odd ones (units are sorted by cost,
-  // so alternating the direction evens out the bias of a fixed stride).  The CTAs that run at the same time thus
-  // work on adjacent units of the same KV head and stream the same K/V tiles: one copy in L2 serves them all.
-  // A round never mixes two round groups, so all its items cost about the same and the CTAs stay in step.
-  // Every role walks the same sequence.
+  // Work order.  Item w = (head within a group of gi heads, unit, group), innermost first; gi = the query heads of
+  // one KV head when the head range is made of whole KV-head groups, else 1.  Units are sorted by cost, so the CTAs
+  // that run at the same time work on adjacent units of the same KV head and stream the same K/V tiles: one copy in
+  // L2 serves them all.  Items are handed out dynamically: the producer thread takes item numbers from a global
+  // counter and passes (unit, head) through a small ring in shared memory to the issuing threads and the softmax
+  // and epilogue warps, which all consume every item in order; -1 ends the list.
   const int gi = a.head_group;
-  const int64_t G = gridDim.x;
-  const int64_t rpg = ((int64_t)a.n_units * a.round_heads + G - 1) / G;      // rounds per (full) round group
-  const int n_round_groups = (a.head_count + a.round_heads - 1) / a.round_heads;
-  const int last_heads = a.head_count - (n_round_groups - 1) * a.round_heads;   // the last group may be smaller
-  auto work_item = [&](int64_t round, const int32_t*& U, int& h) -> bool {
-    const int gidx = (int)min(round / rpg, (int64_t)(n_round_groups - 1));
-    const int64_t rr = round - (int64_t)gidx * rpg;
-    const int64_t idx = rr * G + ((rr & 1) ? G - 1 - (int64_t)blockIdx.x : (int64_t)blockIdx.x);
-    const int hcnt = min(a.round_heads, a.head_count - gidx * a.round_heads);
-    if (idx >= (int64_t)a.n_units * hcnt) return false;       // padding at the end of a round group
-    const int64_t t = idx / gi;
-    U = a.units + (size_t)(t % a.n_units) * FCP_FWD_UNIT_W;
-    h = a.head_begin + gidx * a.round_heads + (int)(t / a.n_units) * gi + (int)(idx % gi);
-    return true;
+  // returns 1 with (U, h) of the next item, 0 at the end of the list, -1 if the CTA is aborting
+  auto take_item = [&](uint32_t& n, const int32_t*& U, int& h, bool whole_warp) -> int {
+    const uint32_t slot = n % FWD_WORK_SLOTS, par = (n / FWD_WORK_SLOTS) & 1;
+    const bool got = whole_warp ? mbar_wait_warp(BAR(B_WFULL + slot), par, wctx, 40) : mbar_wait(BAR(B_WFULL + slot), par, wctx, 40);
+    if (!got) return -1;
+    const int unit = work_ring[2 * slot];
+    h = work_ring[2 * slot + 1];
+    if (whole_warp) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(BAR(B_WEMPTY + slot));
+    } else {
+      mbar_arrive(BAR(B_WEMPTY + slot));
+    }
+    ++n;
+    if (unit < 0) return 0;
+    U = a.units + (size_t)unit * FCP_FWD_UNIT_W;
+    return 1;
   };
-  const int64_t n_rounds = rpg * (n_round_groups - 1) + ((int64_t)a.n_units * last_heads + G - 1) / G;
 
   if (warp < 4) asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_CTRL ";");
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t kv_it = 0, qcnt[2] = {0, 0};
+      uint32_t kv_it = 0, qcnt[2] = {0, 0}, nw = 0;
       bool ok = true;
 #pragma unroll 1
-      uint32_t sync_misses = 0;
-      for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
-        // Meeting point of the grid at the start of a round.  When one KV head's keys and values exceed the L2
-        // the CTAs only share K/V tiles while they sweep them in step; small differences in speed add up over
-        // hundreds of rounds, so they wait for each other here.  The wait is advisory: nothing depends on it,
-        // it ends after round_sync_ns whoever is missing, and a CTA that ran out of patience four times stops
-        // waiting for the rest of the launch.
-        if (a.round_counter != nullptr && sync_misses < 4) {
-          atomicAdd(a.round_counter, 1);
-          const int target = (int)((rnd + 1) * G);
-          const uint32_t t0 = globaltimer_lo();
-          bool met = true;
-          while (*(volatile int32_t*)a.round_counter < target) {
-            if (globaltimer_lo() - t0 > a.round_sync_ns) { met = false; break; }
-            __nanosleep(200);
-          }
-          if (!met) ++sync_misses;
+      while (ok) {
+        const int64_t w = atomicAdd(a.work_counter, 1);
+        const uint32_t slot = nw % FWD_WORK_SLOTS;
+        ok = mbar_wait(BAR(B_WEMPTY + slot), ((nw / FWD_WORK_SLOTS) & 1) ^ 1, wctx, 41);
+        if (!ok) break;
+        const bool last = w >= n_work;
+        int unit = -1, h = 0;
+        if (!last) {
+          const int64_t t = w / gi;
+          unit = (int)(t % a.n_units);
+          h = a.head_begin + (int)(t / a.n_units) * gi + (int)(w % gi);
         }
-        const int32_t* U;
-        int h;
-        if (!work_item(rnd, U, h)) continue;
+        work_ring[2 * slot] = unit;
+        work_ring[2 * slot + 1] = h;
+        mbar_arrive(BAR(B_WFULL + slot));      // release: the two stores above are visible to the waiters
+        ++nw;
+        if (last) break;
+        const int32_t* U = a.units + (size_t)unit * FCP_FWD_UNIT_W;
         const int hk = h / g;
         const int nt[2] = {__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1)};
         const int q_row0 = __ldg(U + FU_Q_ROW0);
@@ -222,13 +225,14 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int s = warp - 1;
       const uint32_t t_s = tmem + S_COL0 + s * 128, t_o = tmem + O_COL0 + s * 128;
       const uint32_t q_addr = sbase + SM::Q_OFF + s * SM::Q_TILE_BYTES;
-      uint32_t kv_it = 0, qcnt = 0, pcnt = 0, ocnt = 0;
+      uint32_t kv_it = 0, qcnt = 0, pcnt = 0, ocnt = 0, nw = 0;
       bool ok = true;
 #pragma unroll 1
-      for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+      while (ok) {
         const int32_t* U;
         int h;
-        if (!work_item(rnd, U, h)) continue;
+        const int r = take_item(nw, U, h, false);
+        if (r <= 0) { ok = r == 0; break; }
         const int nts = __ldg(U + FU_NT_STAGE0 + s);
         const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
         if (nts > 0) {
@@ -283,13 +287,14 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const uint32_t t_o = tmem_addr(tmem, rb * 32, O_COL0 + s * 128);
     float* stat = (float*)(smem + SM::STAT_OFF) + s * 256;
     const float c2 = a.scale_log2;
-    uint32_t scnt = 0, ucnt = 0, tcnt = 0;
+    uint32_t scnt = 0, ucnt = 0, tcnt = 0, nw = 0;
     bool ok = true;
 #pragma unroll 1
-    for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+    while (ok) {
       const int32_t* U;
       int h;
-      if (!work_item(rnd, U, h)) continue;
+      const int r = take_item(nw, U, h, true);
+      if (r <= 0) { ok = r == 0; break; }
       const int nts = __ldg(U + FU_NT_STAGE0 + s);
       const int n_max = max(__ldg(U + FU_NT_STAGE0), __ldg(U + FU_NT_STAGE1));
       const int q_pos = __ldg(U + FU_Q_ROW0) + s * 128 + row;
@@ -414,13 +419,14 @@ fcp_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     asm volatile("setmaxnreg.dec.sync.aligned.u32 " FCP_FWD_REGS_EPI ";");
     const int rb = warp & 3;
     const int row = rb * 32 + lane;
-    uint32_t ecnt0 = 0, ecnt1 = 0;             // phases seen per Q tile
+    uint32_t ecnt0 = 0, ecnt1 = 0, nw = 0;     // phases seen per Q tile; work items taken
     bool ok = true;
 #pragma unroll 1
-    for (int64_t rnd = 0; rnd < n_rounds && ok; ++rnd) {
+    while (ok) {
       const int32_t* U;
       int h;
-      if (!work_item(rnd, U, h)) continue;
+      const int r = take_item(nw, U, h, true);
+      if (r <= 0) { ok = r == 0; break; }
       const int hl = h - a.head_begin;
       const int q_rows = __ldg(U + FU_Q_ROWS);
       const int64_t prow0 = (int64_t)__ldg(U + FU_PART_ROW0);

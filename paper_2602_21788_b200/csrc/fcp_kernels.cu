@@ -2,7 +2,6 @@
 // preprocess, dQ conversion) and the glue around the tensor-core kernels of fcp_fwd.cuh and
 // fcp_bwd.cuh.  No call here allocates device memory except fcp_plan_upload.
 #include <cstdio>
-#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -399,28 +398,9 @@ int launch_fwd(const fcp_plan* plan, const void* q, const void* k, const void* v
   const int grid = (int)std::min<int64_t>(n_work, plan->sm_count);
   if (grid == 0) return FCP_OK;
   cudaStream_t st = (cudaStream_t)stream;
-  {
-    // Where one KV head's K and V of the longest sequence exceed what the 126 MB L2 can hold next to everything
-    // else (above ~96 MB), the CTAs only share K/V tiles while they sweep them in step.  There the heads are
-    // dealt out in round groups of whole KV-head groups (as many as it takes to fill at least 16 rounds), so that
-    // a round never mixes the cheap tail of one KV head with the expensive head of the next, and the grid meets
-    // at every round start.  Measured on the forward pass alone: 201 MB per KV head (`extreme_512k`) 2.50 s ->
-    // 2.36 s; at 67 MB the waiting costs 2 %, and on batches of many medium sequences the padding of the round
-    // groups costs 2-4 %, so everywhere else all heads form one group and nobody waits.
-    int sync = -1;
-    if (const char* e = getenv("FCP_FWD_ROUND_SYNC")) sync = atoi(e);       // debug override: 0 off, 1 on
-    if (sync < 0) sync = (int64_t)plan->max_seqlen * P.head_dim * 4 > (int64_t(96) << 20);
-    a.round_heads = head_count;
-    a.round_counter = nullptr;
-    a.round_sync_ns = 500000u;
-    if (sync && grid > 1) {
-      const int64_t per_kv = (int64_t)a.n_units * a.head_group;
-      const int64_t m = std::min<int64_t>(head_count / a.head_group, std::max<int64_t>(1, (16LL * grid + per_kv - 1) / per_kv));
-      a.round_heads = (int32_t)m * a.head_group;
-      a.round_counter = plan->d_status + 17;
-      FCP_CUDA_CHECK(cudaMemsetAsync(a.round_counter, 0, sizeof(int32_t), st));
-    }
-  }
+  // the grid's work counter (the status block's word 17; word 16 is the backward grid's)
+  a.work_counter = plan->d_status + 17;
+  FCP_CUDA_CHECK(cudaMemsetAsync(a.work_counter, 0, sizeof(int32_t), st));
   ProfScope prof(plan, 0, st);
   if (P.head_dim == 128)
     fcp_fwd_kernel<128><<<grid, FWD_THREADS, FwdSmem<128>::DYN_BYTES, st>>>(tq, tk, tv, a);

@@ -495,28 +495,3 @@ def test_dk_dv_columns_at_chunk_boundaries_mid_sequence(L, d):
         for j in cols:                                 # each boundary column (and row of dq) on its own
             err = np.linalg.norm(res[name][j] - ref[j])
             assert err <= GRAD_REL * np.linalg.norm(ref[j]), (name, j, err / np.linalg.norm(ref[j]))
-
-
-@pytest.mark.parametrize("lens,degs,hq,hkv,D", [([1000], [7], 8, 1, 128), ([777, 64, 1500], [3, 1, 6], 4, 4, 64),
-                                                ([5000, 300, 2049, 129], [5, 1, 2, 1], 16, 2, 128)])
-def test_round_groups_with_grid_meeting_give_the_same_bits(lens, degs, hq, hkv, D, monkeypatch):
-    """For sequences whose keys exceed the L2 the forward grid deals the heads out in round groups and meets at
-    every round start (an advisory, time-limited wait).  That only changes which CTA runs which item and when:
-    forced on here at small sizes (FCP_FWD_ROUND_SYNC=1, a debug switch), the output bits must not change, for
-    whole KV-head groups and for head passes that split them."""
-    from paper_2602_21788_b200.runner import run_fwd_bwd
-    w = _wl(lens, degs, hq, hkv, D, seed=21)
-    q, k, v = w.tensors(with_do=False)
-    monkeypatch.setenv("FCP_FWD_ROUND_SYNC", "0")
-    a = run_fwd_bwd(w, q, k, v, None, fused=True)
-    monkeypatch.setenv("FCP_FWD_ROUND_SYNC", "1")
-    b = run_fwd_bwd(w, q, k, v, None, fused=True)
-    c = run_fwd_bwd(w, q, k, v, None, fused=True, heads_per_pass=3)
-    p = run_fwd_bwd(w, q, k, v, None)                       # the partial path runs the same kernel
-    monkeypatch.setenv("FCP_FWD_ROUND_SYNC", "0")
-    p0 = run_fwd_bwd(w, q, k, v, None)
-    for x in (b, c):
-        assert np.array_equal(a["o"], x["o"]) and np.array_equal(a["lse"], x["lse"]) and np.array_equal(a["o_f32"], x["o_f32"])
-    assert np.array_equal(p["o"], p0["o"]) and np.array_equal(p["lse"], p0["lse"])
-    o_ref, lse_ref = A.attention_fwd_packed(f64(q), f64(k), f64(v), w.cu_seqlens)
-    assert np.abs(b["o_f32"] - o_ref).max() <= O_MAX and np.abs(b["lse"] - lse_ref).max() <= LSE_MAX
