@@ -2,7 +2,8 @@
 // causal mask k_pos <= q_pos), one persistent grid for all virtual ranks of all sequences.
 //
 // Work unit = (two adjacent 128-row Q tiles of one plan item, one query head).  Roles per CTA:
-//   warp 0        TMA producer: Q tiles and the K/V tile ring (128-byte swizzled boxes)
+//   warp 0        work scheduler (global counter -> shared-memory ring) and TMA producer: Q tiles and the K/V tile
+//                 ring (128-byte swizzled boxes)
 //   warps 1, 2    UMMA issuers, one per Q tile: S = Q K^T into TMEM, O += P V with P read from TMEM
 //   warps 4..7    softmax for Q tile 0: one thread per query row, the whole 128-column row in registers
 //   warps 8..11   softmax for Q tile 1
