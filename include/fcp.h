@@ -19,7 +19,7 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Compute calls only
  *     enqueue work on it; they do not synchronise and do not allocate device memory.
  *   - Calls that use one plan must be stream-ordered with respect to each other: the plan's device
- *     copy holds the status words and the work counter of the backward grid, so two compute calls
+ *     copy holds the status words and the work counters of the forward and backward grids, so two compute calls
  *     on the same plan that overlap on the GPU (different streams, different threads) race.  Use
  *     one plan per concurrent stream.
  *   - The device status words are sticky: once a kernel has recorded FCP_ERR_TIMEOUT they keep it
