@@ -246,8 +246,9 @@ int fcp_attn_bwd_heads(const fcp_plan* plan, const void* q, const void* k, const
  * caller-owned DEVICE buffer of `workspace_bytes` >= fcp_host_workspace_bytes(plan); host pointers
  * should be pinned for the copies to be asynchronous.
  * The batch is cut into up to 8 runs of consecutive sequences (packed tensors are token-major, so a
- * run is one contiguous slice of every tensor); the inputs of the next run come in and the results
- * of the previous one go out while the kernels of the current run execute (two internal copy
+ * run is one contiguous slice of every tensor), and a run of several hundred megabytes further into
+ * passes over whole KV heads (strided slices); the inputs of the next slice come in and the results
+ * of the previous one go out while the kernels of the current slice execute (two internal copy
  * streams, ordered after the work already queued on `stream`).  The first call on a plan is the
  * one exception to "compute calls do not allocate": it builds and uploads the plans of the runs
  * and creates the copy streams and events (small allocations, all released by fcp_plan_destroy).

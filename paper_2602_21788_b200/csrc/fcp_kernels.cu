@@ -689,9 +689,19 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
     b0 = b1;
   }
   tok0.push_back(T);
-  // streams and events: [0] start, [1] last copy out, then per group (q, k, v up; dO up; forward done; backward done)
+  // A group whose query tensor alone is hundreds of megabytes (one very long sequence) is additionally cut into
+  // passes over whole KV heads, so that its copies overlap its own kernels too: at least ~256 MB of q per pass.
+  std::vector<int32_t> passes;
+  int64_t total_passes = 0;
+  for (size_t g = 0; g < groups.size(); ++g) {
+    const int64_t q_bytes = (tok0[g + 1] - tok0[g]) * plan->params.hq * plan->params.head_dim * 2;
+    const int32_t np = (int32_t)std::max<int64_t>(1, std::min<int64_t>(plan->params.hkv, q_bytes / (int64_t(256) << 20)));
+    passes.push_back(np);
+    total_passes += np;
+  }
+  // streams and events: [0] start, [1] last copy out, then per (group, pass): q, k, v up; dO up; forward done; backward done
   cudaStream_t in = nullptr, out = nullptr;
-  std::vector<void*> ev(2 + 4 * groups.size(), nullptr);
+  std::vector<void*> ev(2 + 4 * (size_t)total_passes, nullptr);
   cudaError_t e = cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking);
   for (size_t i = 0; i < ev.size() && e == cudaSuccess; ++i) {
@@ -711,6 +721,7 @@ int build_host_groups(const fcp_plan* plan, void* stream) {
   plan->host_events = std::move(ev);
   plan->groups = std::move(groups);
   plan->group_tok0 = std::move(tok0);
+  plan->group_passes = std::move(passes);
   return FCP_OK;
 }
 
@@ -756,46 +767,64 @@ extern "C" int fcp_attn_fwd_bwd_host(const fcp_plan* plan, const void* q_host, c
   // complete when this call returns.
   cudaStream_t s_in = (cudaStream_t)plan->host_in, s_out = (cudaStream_t)plan->host_out;
   auto EV = [&](int i) { return (cudaEvent_t)plan->host_events[i]; };
-  auto ev_qkv = [&](int g) { return EV(2 + 4 * g); };
-  auto ev_do = [&](int g) { return EV(3 + 4 * g); };
-  auto ev_fwd = [&](int g) { return EV(4 + 4 * g); };
-  auto ev_bwd = [&](int g) { return EV(5 + 4 * g); };
+  // Work is cut twice: into groups (runs of consecutive sequences: contiguous token slices) and, for large groups,
+  // into passes over whole KV heads with their query heads (strided slices of every token row: 2-D copies).  The
+  // forward pass of a slice needs q, k, v only: dO follows them and arrives while the forward kernel runs; o and
+  // lse leave while the backward kernels run (they only read them).
+  struct Slice { int g, hk0, hkc, ev0; };
+  std::vector<Slice> slices;
+  {
+    int ev0 = 2;
+    for (int g = 0; g < G; ++g) {
+      const int np = plan->group_passes[g];
+      const int per = (P.hkv + np - 1) / np;
+      for (int hk0 = 0; hk0 < P.hkv; hk0 += per, ev0 += 4) slices.push_back(Slice{g, hk0, std::min(per, P.hkv - hk0), ev0});
+    }
+  }
+  const int gq = P.hq / P.hkv;
   HostDrain drain{s_in, s_out, st};
   FCP_CUDA_CHECK(cudaEventRecord(EV(0), st));
   FCP_CUDA_CHECK(cudaStreamWaitEvent(s_in, EV(0), 0));
   FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, EV(0), 0));
-  // The forward pass of a run needs q, k, v only: dO follows them and arrives while the forward kernel runs;
-  // o and lse leave while the backward kernels run (they only read them).
-  for (int g = 0; g < G; ++g) {
-    const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.q + t0 * rq, (const char*)q_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.k + t0 * rkv, (const char*)k_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.v + t0 * rkv, (const char*)v_host + t0 * rkv, nt * rkv, cudaMemcpyHostToDevice, s_in));
-    FCP_CUDA_CHECK(cudaEventRecord(ev_qkv(g), s_in));
-    FCP_CUDA_CHECK(cudaMemcpyAsync(w + L.d_o + t0 * rq, (const char*)d_o_host + t0 * rq, nt * rq, cudaMemcpyHostToDevice, s_in));
-    FCP_CUDA_CHECK(cudaEventRecord(ev_do(g), s_in));
+  // copies of the heads [h0, h0 + hc) of nt token rows: width hc * bytes per head, pitch = the row of all heads
+  auto copy_heads = [&](char* dst, const char* src, int64_t t0, int64_t nt, int64_t row_bytes, int64_t head_bytes, int h0, int hc,
+                        cudaMemcpyKind kind, cudaStream_t cs) {
+    return cudaMemcpy2DAsync(dst + t0 * row_bytes + h0 * head_bytes, (size_t)row_bytes, src + t0 * row_bytes + h0 * head_bytes,
+                             (size_t)row_bytes, (size_t)(hc * head_bytes), (size_t)nt, kind, cs);
+  };
+  const int64_t hb = D * 2;   // bytes of one head of one token (bf16)
+  for (const Slice& sl : slices) {
+    const int64_t t0 = plan->group_tok0[sl.g], nt = plan->group_tok0[sl.g + 1] - t0;
+    const int h0 = sl.hk0 * gq, hc = sl.hkc * gq;
+    FCP_CUDA_CHECK(copy_heads(w + L.q, (const char*)q_host, t0, nt, rq, hb, h0, hc, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(copy_heads(w + L.k, (const char*)k_host, t0, nt, rkv, hb, sl.hk0, sl.hkc, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(copy_heads(w + L.v, (const char*)v_host, t0, nt, rkv, hb, sl.hk0, sl.hkc, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaEventRecord(EV(sl.ev0), s_in));
+    FCP_CUDA_CHECK(copy_heads(w + L.d_o, (const char*)d_o_host, t0, nt, rq, hb, h0, hc, cudaMemcpyHostToDevice, s_in));
+    FCP_CUDA_CHECK(cudaEventRecord(EV(sl.ev0 + 1), s_in));
   }
-  for (int g = 0; g < G; ++g) {
-    const fcp_plan* sub = plan->groups[g];
-    const int64_t t0 = plan->group_tok0[g], nt = plan->group_tok0[g + 1] - t0;
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_qkv(g), 0));
-    if ((rc = fcp_attn_fwd_fused(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, 0, P.hq, w + L.o + t0 * rq,
+  for (const Slice& sl : slices) {
+    const fcp_plan* sub = plan->groups[sl.g];
+    const int64_t t0 = plan->group_tok0[sl.g], nt = plan->group_tok0[sl.g + 1] - t0;
+    const int h0 = sl.hk0 * gq, hc = sl.hkc * gq;
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, EV(sl.ev0), 0));
+    if ((rc = fcp_attn_fwd_fused(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, h0, hc, w + L.o + t0 * rq,
                                  nullptr, (float*)(w + L.lse + t0 * rl), st)) != FCP_OK)
       return rc;
-    FCP_CUDA_CHECK(cudaEventRecord(ev_fwd(g), st));
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_fwd(g), 0));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)o_host + t0 * rq, w + L.o + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)lse_host + t0 * rl, w + L.lse + t0 * rl, nt * rl, cudaMemcpyDeviceToHost, s_out));
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, ev_do(g), 0));
-    if ((rc = fcp_attn_bwd(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, w + L.o + t0 * rq,
-                           w + L.d_o + t0 * rq, (float*)(w + L.lse + t0 * rl), w + L.dq + t0 * rq, w + L.dk + t0 * rkv,
-                           w + L.dv + t0 * rkv, w + L.scratch, bwd_scratch_need(sub, P.hkv), st)) != FCP_OK)
+    FCP_CUDA_CHECK(cudaEventRecord(EV(sl.ev0 + 2), st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, EV(sl.ev0 + 2), 0));
+    FCP_CUDA_CHECK(copy_heads((char*)o_host, w + L.o, t0, nt, rq, hb, h0, hc, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(copy_heads((char*)lse_host, w + L.lse, t0, nt, rl, 4, h0, hc, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(st, EV(sl.ev0 + 1), 0));
+    if ((rc = fcp_attn_bwd_heads(sub, w + L.q + t0 * rq, w + L.k + t0 * rkv, w + L.v + t0 * rkv, w + L.o + t0 * rq,
+                                 w + L.d_o + t0 * rq, (float*)(w + L.lse + t0 * rl), sl.hk0, sl.hkc, w + L.dq + t0 * rq,
+                                 w + L.dk + t0 * rkv, w + L.dv + t0 * rkv, w + L.scratch, bwd_scratch_need(sub, sl.hkc), st)) != FCP_OK)
       return rc;
-    FCP_CUDA_CHECK(cudaEventRecord(ev_bwd(g), st));
-    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, ev_bwd(g), 0));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dq_host + t0 * rq, w + L.dq + t0 * rq, nt * rq, cudaMemcpyDeviceToHost, s_out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dk_host + t0 * rkv, w + L.dk + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));
-    FCP_CUDA_CHECK(cudaMemcpyAsync((char*)dv_host + t0 * rkv, w + L.dv + t0 * rkv, nt * rkv, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(cudaEventRecord(EV(sl.ev0 + 3), st));
+    FCP_CUDA_CHECK(cudaStreamWaitEvent(s_out, EV(sl.ev0 + 3), 0));
+    FCP_CUDA_CHECK(copy_heads((char*)dq_host, w + L.dq, t0, nt, rq, hb, h0, hc, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(copy_heads((char*)dk_host, w + L.dk, t0, nt, rkv, hb, sl.hk0, sl.hkc, cudaMemcpyDeviceToHost, s_out));
+    FCP_CUDA_CHECK(copy_heads((char*)dv_host, w + L.dv, t0, nt, rkv, hb, sl.hk0, sl.hkc, cudaMemcpyDeviceToHost, s_out));
   }
   FCP_CUDA_CHECK(cudaEventRecord(EV(1), s_out));
   FCP_CUDA_CHECK(cudaStreamWaitEvent(st, EV(1), 0));

@@ -58,7 +58,8 @@ struct fcp_plan {
   mutable std::vector<int64_t> group_tok0;   // first packed token of each group, plus T at the end
   mutable void* host_in = nullptr;           // cudaStream_t: host -> device copies of the host entry point
   mutable void* host_out = nullptr;          // cudaStream_t: device -> host copies
-  mutable std::vector<void*> host_events;    // cudaEvent_t: start, last copy out, then (inputs up, kernels done) per group
+  mutable std::vector<int32_t> group_passes; // KV-head passes of each group (large groups are also pipelined by KV head)
+  mutable std::vector<void*> host_events;    // cudaEvent_t: start, last copy out, then four per (group, pass)
 
   // optional kernel timing: ring of event pairs per kernel kind (void* = cudaEvent_t)
   bool profiling = false;

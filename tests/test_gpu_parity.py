@@ -295,6 +295,38 @@ def test_host_buffer_entry_point_matches_device_path(lens, degs):
     assert e.value.status == fcp.FCP_ERR_WORKSPACE
 
 
+def test_host_buffer_entry_point_pipelines_a_long_sequence_by_kv_heads():
+    """A group whose q slice exceeds 512 MB is also cut into passes over whole KV heads (strided 2-D copies, the
+    forward by head range, the backward by KV-head range): same results as the device path, bit for bit where
+    that path is deterministic."""
+    from paper_2602_21788_b200 import fcp
+    from paper_2602_21788_b200.runner import DeviceState
+    w = _wl([61440, 4096], [5, 1], 40, 8, 128, seed=8)
+    q, k, v, do = w.device_tensors()
+    ds = DeviceState(w, q, k, v, do, partials=False)
+    ds.forward_fused()
+    ds.backward()
+    torch.cuda.synchronize()
+    ds.check_status()
+    T, hq, hkv, D = w.total_tokens, w.hq, w.hkv, w.head_dim
+    pin = lambda t: t.view(torch.int16).cpu().pin_memory()
+    hq_, hk_, hv_, hdo_ = pin(q), pin(k), pin(v), pin(do)
+    ho = torch.zeros((T, hq, D), dtype=torch.int16).pin_memory()
+    hdq = torch.zeros((T, hq, D), dtype=torch.int16).pin_memory()
+    hdk = torch.zeros((T, hkv, D), dtype=torch.int16).pin_memory()
+    hdv = torch.zeros((T, hkv, D), dtype=torch.int16).pin_memory()
+    hlse = torch.zeros((T, hq), dtype=torch.float32).pin_memory()
+    nbytes = ds.plan.host_workspace_bytes()
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    fcp.fcp_attn_fwd_bwd_host(ds.plan, hq_, hk_, hv_, hdo_, ho, hlse, hdq, hdk, hdv, ws, nbytes,
+                              torch.cuda.current_stream().cuda_stream)
+    assert ds.plan.device_status()[0] == 0
+    assert torch.equal(ho, ds.o.view(torch.int16).cpu()) and torch.equal(hlse, ds.lse.cpu())
+    assert torch.equal(hdk, ds.dk.view(torch.int16).cpu()) and torch.equal(hdv, ds.dv.view(torch.int16).cpu())
+    a, b = hdq.view(torch.bfloat16).float(), ds.dq.float().cpu()
+    assert torch.isfinite(a).all() and (a - b).norm() <= 1e-2 * b.norm()
+
+
 def test_workspace_too_small_is_reported():
     from paper_2602_21788_b200 import fcp
     from paper_2602_21788_b200.runner import DeviceState
