@@ -87,3 +87,61 @@ def test_rows_outside_spans_keep_their_causal_bits_and_partial_path_refuses_span
         ds.forward()
     assert e.value.status == fcp.FCP_ERR_UNSUPPORTED
     torch.cuda.synchronize()
+
+
+@pytest.mark.slow
+def test_full_size_bimodal_with_image_spans_sampled():
+    """The benchmark's span workload at its real shape (131 072 tokens, 32 heads, 80 spans of 256-2048 tokens):
+    sampled forward rows and dQ rows, inside spans, at their edges and outside, against the oracle's single-row
+    form (a row with limit lim sees exactly what the causal row lim - 1 sees), plus dK/dV columns at the very end of
+    the longest sequence."""
+    import math
+    from oracle import attention_ref as A
+    from paper_2602_21788_b200.runner import DeviceState
+    w = synth.make_workload("bimodal_128k_spans", 0)
+    q, k, v, do = w.device_tensors()
+    ds = DeviceState(w, q, k, v, do, partials=False, want_o_f32=True)
+    ds.forward_fused()
+    ds.backward()
+    torch.cuda.synchronize()
+    ds.check_status()
+    b64 = lambda t: t.float().cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(0)
+    cu, D = w.cu_seqlens, w.head_dim
+    long_seqs = [b for b in range(len(w.seqlens)) if w.spans[b]]
+    o_err, l_err, num, den = [], [], 0.0, 0.0
+    for n in range(40):
+        b = long_seqs[n % len(long_seqs)]
+        L, t0 = int(w.seqlens[b]), int(cu[b])
+        lim = S.row_limits(L, w.spans[b])
+        a_, e_ = w.spans[b][int(rng.integers(len(w.spans[b])))]
+        i = [a_, e_ - 1, int(rng.integers(a_, e_)), max(0, a_ - 1), min(L - 1, e_), int(rng.integers(L))][n % 6]
+        h = int(rng.integers(w.hq))
+        ks, vs = b64(k[t0:t0 + int(lim[i]), h]), b64(v[t0:t0 + int(lim[i]), h])      # hq == hkv in this workload
+        qi, doi = b64(q[t0 + i, h]), b64(do[t0 + i, h])
+        o_ref, lse_ref = A.attention_row(qi, ks, vs, int(lim[i]) - 1)
+        dq_ref, _, _ = A.attention_row_grad(qi, ks, vs, doi, int(lim[i]) - 1)
+        o_err.append(np.abs(ds.o_f32[t0 + i, h].cpu().numpy().astype(np.float64) - o_ref))
+        l_err.append(abs(float(ds.lse[t0 + i, h]) - lse_ref))
+        num += np.sum((b64(ds.dq[t0 + i, h]) - dq_ref) ** 2)
+        den += np.sum(dq_ref ** 2)
+    o_err = np.concatenate(o_err)
+    assert o_err.max() <= O_MAX and o_err.mean() <= O_MEAN and max(l_err) <= LSE_MAX
+    assert math.sqrt(num / den) <= GRAD_REL
+    # dK/dV of the last 8 tokens of the longest sequence: every row from the first query that sees them on
+    b = int(np.argmax(w.seqlens))
+    L, t0 = int(w.seqlens[b]), int(cu[b])
+    lim, first = S.row_limits(L, w.spans[b]), S.first_queries(L, w.spans[b])
+    j0, hk = L - 8, 3
+    ks, vs = b64(k[t0:t0 + L, hk]), b64(v[t0:t0 + L, hk])
+    dk_ref, dv_ref = np.zeros((8, D)), np.zeros((8, D))
+    for i in range(int(first[j0]), L):
+        qi, doi = b64(q[t0 + i, hk]), b64(do[t0 + i, hk])
+        n_i = int(lim[i])
+        _, p, dsr = A.attention_row_grad(qi, ks[:n_i], vs[:n_i], doi, n_i - 1)
+        lo = max(j0, 0)
+        if n_i > lo:
+            dv_ref[: n_i - lo] += p[lo:, None] * doi[None, :]
+            dk_ref[: n_i - lo] += dsr[lo:, None] * qi[None, :] / math.sqrt(D)
+    for name, ref, got in (("dk", dk_ref, ds.dk), ("dv", dv_ref, ds.dv)):
+        assert np.linalg.norm(b64(got[t0 + j0:t0 + L, hk]) - ref) <= GRAD_REL * np.linalg.norm(ref), name
